@@ -1,0 +1,156 @@
+/*
+ * sol_attn.h -- C ABI of the B200 (sm_100a) Sol-Attn forward path.
+ *
+ * Sol-Attn ("on-the-fly attention sparsification") computes, for every query block i of a
+ * head, softmax attention in which key/value blocks whose pooled proxy score exceeds a
+ * query-dependent threshold are processed exactly and all other blocks are folded in through
+ * their pooled key and summed value, all inside one online-softmax pass.
+ *
+ * Conventions shared by every entry point
+ *   - q, k, v, out: DEVICE pointers to contiguous row-major [B, H, N, d] bf16 tensors,
+ *     16-byte aligned.  N is the number of tokens per (batch, head) (the paper's L).
+ *   - Every logit is multiplied by scale = 1/sqrt(d) unless the _ex call overrides it.
+ *   - `threshold` is the standardized cutoff beta of Eq. (4): tau_i = mu_i + beta*sigma_i.
+ *     +INFINITY routes nothing to the exact branch, -INFINITY routes everything.
+ *   - The library owns no device memory, creates no stream and never synchronises unless
+ *     stated.  All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) and the call returns after the last launch.  Errors that the
+ *     host can see (bad pointers, unsupported shapes, too-small workspace, wrong GPU
+ *     architecture) are returned before anything is launched.  Errors found on the device
+ *     (a bounded wait that expired) are recorded in a status word inside the workspace and
+ *     read back with sol_attn_read_device_status().
+ *   - Scratch memory is a caller-allocated device workspace of sol_attn_workspace_bytes()
+ *     bytes, 1024-byte aligned, attached with sol_attn_bind_workspace() (process-wide, one at
+ *     a time; not thread-safe) or passed per call through sol_attn_args.  Its contents are
+ *     overwritten by every call.  Calls that share a workspace and overlap on the GPU race.
+ *   - Supported shapes: d in {64, 128}; block_q == block_k in {64, 128} for the fused
+ *     kernels (the pooling pre-pass accepts any block size in [1, 1024]); B, H, N >= 1;
+ *     ceil(N / block_k) <= 65535.  Anything else returns SOL_ERR_UNSUPPORTED_SHAPE.
+ */
+#ifndef SOL_ATTN_H_
+#define SOL_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t sol_status_t;
+typedef void*   sol_stream_t;   /* a cudaStream_t */
+
+enum {
+  SOL_OK                    =  0,
+  SOL_ERR_INVALID_ARG       = -1,  /* NULL / misaligned pointer, non-positive size, NaN threshold */
+  SOL_ERR_UNSUPPORTED_SHAPE = -2,  /* d, block sizes or N outside the supported set            */
+  SOL_ERR_UNSUPPORTED_ARCH  = -3,  /* current device is not compute capability 10.x            */
+  SOL_ERR_WORKSPACE         = -4,  /* no workspace bound / workspace too small or misaligned   */
+  SOL_ERR_CUDA              = -5,  /* a CUDA runtime or driver call failed (launch, tensor map)*/
+  SOL_ERR_DEVICE_TIMEOUT    = -6   /* a bounded device-side wait expired; output is invalid    */
+};
+
+/* what the fused kernel computes */
+enum {
+  SOL_MODE_SOL        = 0,  /* Algorithm 1: exact branch + proxy-score-reuse approximation     */
+  SOL_MODE_DENSE      = 1,  /* Eq. (1): every block exact, no routing                          */
+  SOL_MODE_EXACT_ONLY = 2   /* Eq. (2): routed blocks exact, unselected blocks dropped         */
+};
+
+/* which implementation of the fused kernel runs */
+enum {
+  SOL_IMPL_AUTO     = 0,  /* tcgen05 kernel when the shape allows it, else the mma.sync one    */
+  SOL_IMPL_TCGEN05  = 1,  /* TMA + tcgen05.mma + TMEM kernel (d = 128, block 128)              */
+  SOL_IMPL_MMA_SYNC = 2   /* portable warp-level mma.sync kernel (all supported shapes)        */
+};
+
+/* Human-readable name of a status code; never NULL, static storage. */
+const char* sol_attn_status_string(sol_status_t status);
+
+/* Bytes of device workspace needed for the given problem (0 if the shape is unsupported).
+ * The workspace holds the pre-attention results of Sec. 3.1-3.2 -- pooled queries Qbar, pooled
+ * keys KC (token mean, Eq. 3), summed values VC (defined before Eq. 9), bf16 operand copies,
+ * pooled-key moments (Eq. 5), mu/sigma/tau per query block (Eq. 4) -- plus a status word. */
+size_t sol_attn_workspace_bytes(int B, int H, int N, int d, int block_q, int block_k);
+
+/* Byte offsets of the parity-relevant arrays inside a workspace laid out for the given problem.
+ * All arrays are fp32 except counts_unused.  qbar: [B,H,Nq,d] mean of each query block;
+ * kc: [B,H,Nk,d] mean of each key block; vc: [B,H,Nk,d] SUM of each value block;
+ * mu, sigma, tau: [B,H,Nq]; status: int32[16] (word 0 = device status, see below). */
+typedef struct {
+  size_t status, qbar, kc, vc, mu, sigma, tau, total_bytes;
+  int32_t n_q_blocks, n_k_blocks;
+} sol_attn_ws_view;
+sol_status_t sol_attn_workspace_view(int B, int H, int N, int d, int block_q, int block_k,
+                                     sol_attn_ws_view* view /* host, out */);
+
+/* Attach a device workspace and (optionally) a device int32 [B, H, ceil(N/block_q)] array that
+ * receives, per query block, the number of key blocks routed to the exact branch (|S_i| of
+ * Eq. 4; overwritten, not accumulated, by every forward).  dev_counts may be NULL.  The size is
+ * checked against each later call's shape.  Passing dev_ws == NULL detaches. */
+sol_status_t sol_attn_bind_workspace(void* dev_ws, size_t bytes, int32_t* dev_counts);
+
+/* Pre-attention pass (Eq. 3 pooling; Eq. 5 moments; Eq. 4 thresholds): one bandwidth-bound
+ * read of q, k, v that fills the bound workspace.  `threshold` is beta.  q may be NULL when
+ * only K/V pooling is wanted (thresholds are then not produced). */
+sol_status_t sol_attn_pool(const void* q, const void* k, const void* v,
+                           int B, int H, int N, int d, int block_q, int block_k,
+                           float threshold, sol_stream_t stream);
+
+/* Algorithm 1 end to end: the pooling pre-pass followed by the fused single-pass kernel
+ * (on-the-fly thresholding, exact branch on routed blocks, approximate branch on the rest,
+ * Eqs. 9-10), using the bound workspace.  Rows >= N of `out` do not exist and are never
+ * written. */
+sol_status_t sol_attn_forward(const void* q, const void* k, const void* v, void* out,
+                              int B, int H, int N, int d, int block_q, int block_k,
+                              float threshold, sol_stream_t stream);
+
+/* Dense softmax attention, Eq. (1), through the same fused kernel with routing off
+ * (block size 128 for d = 128, 64 for d = 64).  counts, when bound, receive ceil(N/block). */
+sol_status_t sol_attn_dense(const void* q, const void* k, const void* v, void* out,
+                            int B, int H, int N, int d, sol_stream_t stream);
+
+/* Fully explicit variant: nothing is taken from the bound state. */
+typedef struct {
+  const void* q; const void* k; const void* v;  /* device, bf16 [B,H,N,d]                       */
+  void*       out;                              /* device, bf16 [B,H,N,d]                       */
+  int32_t B, H, N, d, block_q, block_k;
+  float   threshold;                            /* beta (ignored in SOL_MODE_DENSE)             */
+  float   scale;                                /* logit scale; <= 0 selects 1/sqrt(d)          */
+  int32_t mode;                                 /* SOL_MODE_*                                   */
+  int32_t impl;                                 /* SOL_IMPL_*                                   */
+  int32_t skip_pool;                            /* 1: reuse the workspace filled by a previous
+                                                   sol_attn_pool / forward of the same q, k, v  */
+  const float* tau_override;                    /* device fp32 [B,H,Nq] raw thresholds replacing
+                                                   mu + beta*sigma (Algorithm 1's own `tau`
+                                                   argument), or NULL                           */
+  void*   workspace; size_t workspace_bytes;    /* device scratch, 1024-byte aligned            */
+  int32_t* counts;                              /* device int32 [B,H,Nq] or NULL                */
+  uint32_t* mask_out;                           /* debug: device bitmask [B,H,Nq,ceil(Nk/32)],
+                                                   bit j%32 of word j/32 set when block j is in
+                                                   S_i; NULL in production (the proxy map is
+                                                   never written to memory otherwise)           */
+  sol_stream_t stream;
+} sol_attn_args;
+sol_status_t sol_attn_forward_ex(const sol_attn_args* args /* host */);
+
+/* End-to-end convenience for callers whose tensors live in HOST memory (pinned memory makes
+ * the copies asynchronous): copies hq, hk, hv into the caller's device staging buffers dq, dk,
+ * dv, runs sol_attn_forward with the bound workspace, copies dout into hout, all on `stream`.
+ * Does not synchronise. */
+sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* hv, void* hout,
+                                   void* dq, void* dk, void* dv, void* dout,
+                                   int B, int H, int N, int d, int block_q, int block_k,
+                                   float threshold, sol_stream_t stream);
+
+/* Synchronises `stream`, then returns the device status word of the bound workspace
+ * (SOL_OK, or SOL_ERR_DEVICE_TIMEOUT when a kernel gave up on a bounded wait) and clears it. */
+sol_status_t sol_attn_read_device_status(sol_stream_t stream);
+
+/* Number of kernels the library has launched since it was loaded (for launch accounting). */
+int64_t sol_attn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SOL_ATTN_H_ */
