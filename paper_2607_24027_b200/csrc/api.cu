@@ -1,0 +1,217 @@
+// C ABI of the Sol-Attn CUDA path: argument validation, workspace bookkeeping, launches.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+
+#include "common.cuh"
+
+namespace {
+
+struct Bound {
+  void* ws = nullptr;
+  size_t bytes = 0;
+  int32_t* counts = nullptr;
+};
+Bound g_bound;
+std::atomic<int64_t> g_launches{0};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+sol_status_t check_arch() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SOL_ERR_CUDA;
+  return major == 10 ? SOL_OK : SOL_ERR_UNSUPPORTED_ARCH;
+}
+
+// Shape checks common to every entry point.  `fused` adds the fused kernels' restrictions.
+sol_status_t check_shape(int B, int H, int N, int d, int block_q, int block_k, bool fused) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || block_q <= 0 || block_k <= 0) return SOL_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if (block_q > 1024 || block_k > 1024) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H > 0x7fffffLL) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if (sol::ceil_div(N, block_k) > 65535 || sol::ceil_div(N, block_q) > 65535) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if (fused && (block_q != block_k || (block_q != 64 && block_q != 128))) return SOL_ERR_UNSUPPORTED_SHAPE;
+  return SOL_OK;
+}
+
+sol::Problem make_problem(int B, int H, int N, int d, int block_q, int block_k, float beta, float scale, int mode) {
+  sol::Problem p{};
+  p.B = B; p.H = H; p.N = N; p.d = d; p.block_q = block_q; p.block_k = block_k;
+  p.BH = B * H;
+  p.Nq = sol::ceil_div(N, block_q);
+  p.Nk = sol::ceil_div(N, block_k);
+  p.scale = scale > 0.f ? scale : 1.0f / std::sqrt((float)d);
+  p.beta = beta;
+  p.mode = mode;
+  return p;
+}
+
+sol_status_t run_pool(const sol::Problem& p, const void* q, const void* k, const void* v, void* ws_base,
+                      cudaStream_t stream) {
+  const sol::WsLayout lay = sol::make_layout(p.BH, p.Nq, p.Nk, p.d);
+  const sol::WsPtrs ws = sol::make_ptrs(ws_base, lay);
+  int n = 0;
+  cudaError_t e = sol::launch_pool(p, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                   static_cast<const __nv_bfloat16*>(v), ws, stream, &n);
+  if (e == cudaSuccess && q) e = sol::launch_thresholds(p, ws, stream, &n);
+  g_launches += n;
+  return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sol_attn_status_string(sol_status_t s) {
+  switch (s) {
+    case SOL_OK: return "SOL_OK";
+    case SOL_ERR_INVALID_ARG: return "SOL_ERR_INVALID_ARG";
+    case SOL_ERR_UNSUPPORTED_SHAPE: return "SOL_ERR_UNSUPPORTED_SHAPE";
+    case SOL_ERR_UNSUPPORTED_ARCH: return "SOL_ERR_UNSUPPORTED_ARCH";
+    case SOL_ERR_WORKSPACE: return "SOL_ERR_WORKSPACE";
+    case SOL_ERR_CUDA: return "SOL_ERR_CUDA";
+    case SOL_ERR_DEVICE_TIMEOUT: return "SOL_ERR_DEVICE_TIMEOUT";
+    default: return "SOL_ERR_UNKNOWN";
+  }
+}
+
+size_t sol_attn_workspace_bytes(int B, int H, int N, int d, int block_q, int block_k) {
+  if (check_shape(B, H, N, d, block_q, block_k, false) != SOL_OK) return 0;
+  return sol::make_layout(B * H, sol::ceil_div(N, block_q), sol::ceil_div(N, block_k), d).total;
+}
+
+sol_status_t sol_attn_workspace_view(int B, int H, int N, int d, int block_q, int block_k, sol_attn_ws_view* view) {
+  if (!view) return SOL_ERR_INVALID_ARG;
+  sol_status_t s = check_shape(B, H, N, d, block_q, block_k, false);
+  if (s != SOL_OK) return s;
+  const int Nq = sol::ceil_div(N, block_q), Nk = sol::ceil_div(N, block_k);
+  const sol::WsLayout w = sol::make_layout(B * H, Nq, Nk, d);
+  view->status = w.status; view->qbar = w.qbar; view->kc = w.kc; view->vc = w.vc;
+  view->mu = w.mu; view->sigma = w.sigma; view->tau = w.tau; view->total_bytes = w.total;
+  view->n_q_blocks = Nq; view->n_k_blocks = Nk;
+  return SOL_OK;
+}
+
+sol_status_t sol_attn_bind_workspace(void* dev_ws, size_t bytes, int32_t* dev_counts) {
+  if (!dev_ws) { g_bound = Bound{}; return SOL_OK; }
+  if ((reinterpret_cast<uintptr_t>(dev_ws) & 1023u) != 0) return SOL_ERR_WORKSPACE;
+  if (bytes < 1024) return SOL_ERR_WORKSPACE;
+  g_bound.ws = dev_ws; g_bound.bytes = bytes; g_bound.counts = dev_counts;
+  return SOL_OK;
+}
+
+sol_status_t sol_attn_pool(const void* q, const void* k, const void* v, int B, int H, int N, int d,
+                           int block_q, int block_k, float threshold, sol_stream_t stream) {
+  sol_status_t s = check_shape(B, H, N, d, block_q, block_k, false);
+  if (s != SOL_OK) return s;
+  if (!k || !v || !aligned16(k) || !aligned16(v) || (q && !aligned16(q)) || std::isnan(threshold))
+    return SOL_ERR_INVALID_ARG;
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  if (g_bound.bytes < sol_attn_workspace_bytes(B, H, N, d, block_q, block_k)) return SOL_ERR_WORKSPACE;
+  if ((s = check_arch()) != SOL_OK) return s;
+  const sol::Problem p = make_problem(B, H, N, d, block_q, block_k, threshold, 0.f, SOL_MODE_SOL);
+  return run_pool(p, q, k, v, g_bound.ws, static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
+  if (!a) return SOL_ERR_INVALID_ARG;
+  sol_status_t s = check_shape(a->B, a->H, a->N, a->d, a->block_q, a->block_k, true);
+  if (s != SOL_OK) return s;
+  if (!a->q || !a->k || !a->v || !a->out) return SOL_ERR_INVALID_ARG;
+  if (!aligned16(a->q) || !aligned16(a->k) || !aligned16(a->v) || !aligned16(a->out)) return SOL_ERR_INVALID_ARG;
+  if (a->mode < SOL_MODE_SOL || a->mode > SOL_MODE_EXACT_ONLY) return SOL_ERR_INVALID_ARG;
+  if (a->impl < SOL_IMPL_AUTO || a->impl > SOL_IMPL_MMA_SYNC) return SOL_ERR_INVALID_ARG;
+  if (a->mode != SOL_MODE_DENSE && !a->tau_override && std::isnan(a->threshold)) return SOL_ERR_INVALID_ARG;
+  if (std::isnan(a->scale) || std::isinf(a->scale)) return SOL_ERR_INVALID_ARG;
+  if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 1023u) != 0) return SOL_ERR_WORKSPACE;
+  if (a->workspace_bytes < sol_attn_workspace_bytes(a->B, a->H, a->N, a->d, a->block_q, a->block_k))
+    return SOL_ERR_WORKSPACE;
+  if ((s = check_arch()) != SOL_OK) return s;
+
+  const sol::Problem p = make_problem(a->B, a->H, a->N, a->d, a->block_q, a->block_k, a->threshold, a->scale, a->mode);
+  int impl = a->impl;
+  if (impl == SOL_IMPL_AUTO) impl = sol::fwd_sm100_supports(p) ? SOL_IMPL_TCGEN05 : SOL_IMPL_MMA_SYNC;
+  if (impl == SOL_IMPL_TCGEN05 && !sol::fwd_sm100_supports(p)) return SOL_ERR_UNSUPPORTED_SHAPE;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(a->stream);
+  const sol::WsLayout lay = sol::make_layout(p.BH, p.Nq, p.Nk, p.d);
+  const sol::WsPtrs ws = sol::make_ptrs(a->workspace, lay);
+  if (cudaMemsetAsync(ws.status, 0, sizeof(int32_t) * sol::kStatusWords, stream) != cudaSuccess) return SOL_ERR_CUDA;
+  if (p.mode != SOL_MODE_DENSE && !a->skip_pool) {
+    s = run_pool(p, a->q, a->k, a->v, a->workspace, stream);
+    if (s != SOL_OK) return s;
+  }
+  const float* tau = a->tau_override ? a->tau_override : ws.tau;
+  int n = 0;
+  cudaError_t e;
+  const auto* q = static_cast<const __nv_bfloat16*>(a->q);
+  const auto* k = static_cast<const __nv_bfloat16*>(a->k);
+  const auto* v = static_cast<const __nv_bfloat16*>(a->v);
+  auto* out = static_cast<__nv_bfloat16*>(a->out);
+  if (impl == SOL_IMPL_TCGEN05) e = sol::launch_fwd_sm100(p, q, k, v, out, ws, tau, a->counts, a->mask_out, stream, &n);
+  else e = sol::launch_fwd_mma_sync(p, q, k, v, out, ws, tau, a->counts, a->mask_out, stream, &n);
+  g_launches += n;
+  return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+}
+
+sol_status_t sol_attn_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int N,
+                              int d, int block_q, int block_k, float threshold, sol_stream_t stream) {
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  sol_attn_args a{};
+  a.q = q; a.k = k; a.v = v; a.out = out;
+  a.B = B; a.H = H; a.N = N; a.d = d; a.block_q = block_q; a.block_k = block_k;
+  a.threshold = threshold; a.scale = 0.f; a.mode = SOL_MODE_SOL; a.impl = SOL_IMPL_AUTO;
+  a.workspace = g_bound.ws; a.workspace_bytes = g_bound.bytes; a.counts = g_bound.counts;
+  a.stream = stream;
+  return sol_attn_forward_ex(&a);
+}
+
+sol_status_t sol_attn_dense(const void* q, const void* k, const void* v, void* out, int B, int H, int N,
+                            int d, sol_stream_t stream) {
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  sol_attn_args a{};
+  a.q = q; a.k = k; a.v = v; a.out = out;
+  a.B = B; a.H = H; a.N = N; a.d = d;
+  a.block_q = a.block_k = (d == 64 ? 64 : 128);
+  a.threshold = 0.f; a.scale = 0.f; a.mode = SOL_MODE_DENSE; a.impl = SOL_IMPL_AUTO;
+  a.workspace = g_bound.ws; a.workspace_bytes = g_bound.bytes; a.counts = g_bound.counts;
+  a.stream = stream;
+  return sol_attn_forward_ex(&a);
+}
+
+sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* hv, void* hout, void* dq, void* dk,
+                                   void* dv, void* dout, int B, int H, int N, int d, int block_q, int block_k,
+                                   float threshold, sol_stream_t stream) {
+  if (!hq || !hk || !hv || !hout || !dq || !dk || !dv || !dout) return SOL_ERR_INVALID_ARG;
+  sol_status_t s = check_shape(B, H, N, d, block_q, block_k, true);
+  if (s != SOL_OK) return s;
+  const size_t bytes = (size_t)B * H * N * d * 2;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(dq, hq, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
+  if (cudaMemcpyAsync(dk, hk, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
+  if (cudaMemcpyAsync(dv, hv, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
+  s = sol_attn_forward(dq, dk, dv, dout, B, H, N, d, block_q, block_k, threshold, stream);
+  if (s != SOL_OK) return s;
+  if (cudaMemcpyAsync(hout, dout, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SOL_ERR_CUDA;
+  return SOL_OK;
+}
+
+sol_status_t sol_attn_read_device_status(sol_stream_t stream) {
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t words[2] = {0, 0};
+  if (cudaMemcpyAsync(words, g_bound.ws, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SOL_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SOL_ERR_CUDA;
+  if (words[0] != 0) {
+    cudaMemsetAsync(g_bound.ws, 0, sizeof(words), st);
+    cudaStreamSynchronize(st);
+    return static_cast<sol_status_t>(words[0]);
+  }
+  return SOL_OK;
+}
+
+int64_t sol_attn_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

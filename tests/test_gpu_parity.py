@@ -1,0 +1,242 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on identical seeded bits."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sol_attn_oracle as orc
+from paper_2607_24027_b200 import synth
+from paper_2607_24027_b200.configs import WORKLOADS, load_betas
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+sb = None
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    global sb
+    from paper_2607_24027_b200 import binding
+    sb = binding
+    sb.lib()
+    yield
+
+
+IMPLS = ["mma_sync", "auto"]
+
+
+def _impl(name):
+    return {"mma_sync": sb.SOL_IMPL_MMA_SYNC, "auto": sb.SOL_IMPL_AUTO, "tcgen05": sb.SOL_IMPL_TCGEN05}[name]
+
+
+def _small_problem(seed, B, H, N, d, structured=True):
+    wl_grid = None
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((3, B, H, N, d)).astype(np.float32)
+    if structured:
+        t = np.linspace(0, 6, N, dtype=np.float32)[:, None] + np.arange(d, dtype=np.float32)[None, :] * 0.37
+        x[0] += 0.8 * np.sin(t)
+        x[1] += 0.8 * np.sin(t)
+    bits = [synth.f32_to_bf16_bits(x[i]) for i in range(3)]
+    return bits
+
+
+def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=0.0, tiles=None):
+    qb, kb, vb = bits
+    q, k, v = (hp.to_dev(x) for x in bits)
+    mode = sb.SOL_MODE_SOL if mode is None else mode
+    out, counts, mask, _ = hp.run_gpu(q, k, v, block, beta, mode=mode, impl=impl, scale=scale)
+    B, H, N, d = q.shape
+    out64 = hp.dev_to_f64(out)
+    agg = {"in_band_flips": 0, "max_abs": 0.0, "rel_l2": 0.0}
+    for b in range(B):
+        for h in range(H):
+            st = hp.check_head(synth.widen(qb[b, h], np.float64), synth.widen(kb[b, h], np.float64),
+                               synth.widen(vb[b, h], np.float64), out64[b, h], mask[b, h],
+                               counts[b, h].cpu().numpy(), block, beta, tiles=tiles,
+                               scale=(scale if scale > 0 else None), mode=mode_name)
+            agg["in_band_flips"] += st["in_band_flips"]
+            agg["max_abs"] = max(agg["max_abs"], st["max_abs"])
+            agg["rel_l2"] = max(agg["rel_l2"], st["rel_l2"])
+    return agg
+
+
+# ----------------------------------------------------------------------------- pre-attention
+@pytest.mark.parametrize("name", ["tiny", "image"])
+def test_pool_and_thresholds(name):
+    wl = WORKLOADS[name]
+    beta = list(load_betas()[name].values())[0]
+    qb, kb, vb = synth.generate(wl)
+    q, k, v = hp.to_dev(qb), hp.to_dev(kb), hp.to_dev(vb)
+    ws = sb.make_workspace(wl.batch, wl.heads, wl.seq_len, wl.d, wl.block, wl.block)
+    sb.sol_attn_bind_workspace(ws)
+    sb.sol_attn_pool(q, k, v, wl.block, wl.block, beta)
+    torch.cuda.synchronize()
+    for h in range(wl.heads):
+        r = orc.routing(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                        synth.widen(vb[0, h], np.float64), wl.block, wl.block, beta)
+        np.testing.assert_allclose(ws.qbar[0, h].cpu().numpy(), r.qbar, rtol=0, atol=2e-6)
+        np.testing.assert_allclose(ws.kc[0, h].cpu().numpy(), r.kc, rtol=0, atol=2e-6)
+        np.testing.assert_allclose(ws.vc[0, h].cpu().numpy(), r.vc, rtol=0, atol=2e-4)
+        np.testing.assert_allclose(ws.mu[0, h].cpu().numpy(), r.mu, rtol=0, atol=2e-5)
+        np.testing.assert_allclose(ws.sigma[0, h].cpu().numpy(), r.sigma, rtol=1e-4, atol=2e-5)
+        np.testing.assert_allclose(ws.tau[0, h].cpu().numpy(), r.tau, rtol=0, atol=5e-5)
+
+
+def test_pool_ragged_and_odd_blocks():
+    bits = _small_problem(3, 2, 3, 1000, 128)
+    qb, kb, vb = bits
+    q, k, v = (hp.to_dev(x) for x in bits)
+    for bq, bk in [(128, 128), (64, 128), (100, 36), (1000, 1)]:
+        ws = sb.make_workspace(2, 3, 1000, 128, bq, bk)
+        sb.sol_attn_bind_workspace(ws)
+        sb.sol_attn_pool(q, k, v, bq, bk, 0.7)
+        torch.cuda.synchronize()
+        for b in range(2):
+            for h in range(3):
+                r = orc.routing(synth.widen(qb[b, h], np.float64), synth.widen(kb[b, h], np.float64),
+                                synth.widen(vb[b, h], np.float64), bq, bk, 0.7)
+                np.testing.assert_allclose(ws.qbar[b, h].cpu().numpy(), r.qbar, rtol=0, atol=2e-6)
+                np.testing.assert_allclose(ws.kc[b, h].cpu().numpy(), r.kc, rtol=0, atol=2e-6)
+                np.testing.assert_allclose(ws.vc[b, h].cpu().numpy(), r.vc, rtol=0, atol=2e-4)
+                np.testing.assert_allclose(ws.tau[b, h].cpu().numpy(), r.tau, rtol=0, atol=5e-5)
+
+
+# ----------------------------------------------------------------------------- fused forward
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_all_tiles(impl):
+    wl = WORKLOADS["tiny"]
+    beta = load_betas()["tiny"][0.3]
+    agg = _check_all_heads(synth.generate(wl), wl.block, beta, _impl(impl))
+    print("tiny", impl, agg)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("rho", [0.2, 0.4, 0.6])
+def test_image_all_tiles(impl, rho):
+    wl = WORKLOADS["image"]
+    beta = load_betas()["image"][rho]
+    agg = _check_all_heads(synth.generate(wl), wl.block, beta, _impl(impl))
+    print("image", impl, rho, agg)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("N,d,block", [(1000, 128, 128), (520, 128, 128), (50, 128, 128), (129, 128, 128),
+                                       (1000, 64, 64), (333, 128, 64), (700, 64, 128)])
+def test_ragged_shapes(impl, N, d, block):
+    bits = _small_problem(N + d, 2, 2, N, d)
+    agg = _check_all_heads(bits, block, 0.4, _impl(impl))
+    print("ragged", impl, N, d, block, agg)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("beta", [-math.inf, math.inf])
+def test_select_all_and_none(impl, beta):
+    bits = _small_problem(11, 1, 2, 900, 128)
+    qb, kb, vb = bits
+    agg = _check_all_heads(bits, 128, beta, _impl(impl))
+    # select-all must also equal dense attention; select-none the pooled-sequence closed form
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out, counts, mask, _ = hp.run_gpu(q, k, v, 128, beta, impl=_impl(impl))
+    nk = mask.shape[-1]
+    assert mask.all() if beta < 0 else not mask.any()
+    assert (counts.cpu().numpy() == (nk if beta < 0 else 0)).all()
+    if beta < 0:
+        for h in range(2):
+            ref = orc.dense_attention(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                                      synth.widen(vb[0, h], np.float64))
+            assert np.abs(hp.dev_to_f64(out)[0, h] - ref).max() <= hp.MAX_ABS
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_dense_mode(impl):
+    bits = _small_problem(12, 1, 3, 777, 128)
+    qb, kb, vb = bits
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out, counts, _, ws = hp.run_gpu(q, k, v, 128, 0.0, mode=sb.SOL_MODE_DENSE, impl=_impl(impl), want_mask=False)
+    assert (counts.cpu().numpy() == ws.view.n_k_blocks).all()
+    o = hp.dev_to_f64(out)
+    for h in range(3):
+        ref = orc.dense_attention(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                                  synth.widen(vb[0, h], np.float64))
+        assert np.abs(o[0, h] - ref).max() <= hp.MAX_ABS
+        assert np.linalg.norm(o[0, h] - ref) / np.linalg.norm(ref) <= hp.REL_L2
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_exact_only_mode_and_scale(impl):
+    bits = _small_problem(13, 1, 2, 1024, 128)
+    _check_all_heads(bits, 128, 0.3, _impl(impl), mode=sb.SOL_MODE_EXACT_ONLY, mode_name="exact_only")
+    _check_all_heads(bits, 128, 0.3, _impl(impl), scale=0.05)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tau_override_and_determinism(impl):
+    bits = _small_problem(14, 1, 2, 1024, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out1, c1, m1, ws = hp.run_gpu(q, k, v, 128, 0.5, impl=_impl(impl))
+    tau = ws.tau.clone()
+    out2, c2, m2, _ = hp.run_gpu(q, k, v, 128, 99.0, impl=_impl(impl), tau_override=tau)
+    assert np.array_equal(m1, m2) and torch.equal(c1, c2)
+    assert torch.equal(out1.view(torch.int16), out2.view(torch.int16))   # run-to-run bit stability
+
+
+# ----------------------------------------------------------------------------- host-side errors
+def test_argument_validation():
+    bits = _small_problem(15, 1, 1, 256, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out = torch.empty_like(q)
+    ws = sb.make_workspace(1, 1, 256, 128, 128, 128)
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 64)
+    assert e.value.status == sb.SOL_ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 32, 32)
+    assert e.value.status == sb.SOL_ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=float("nan"))
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
+    small = sb.make_workspace(1, 1, 256, 128, 128, 128)
+    small.buf = small.buf[:small.buf.numel() - 2048]
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q, k, v, out, small, 128, 128)
+    assert e.value.status == sb.SOL_ERR_WORKSPACE
+    sb.sol_attn_bind_workspace(None)
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward(q, k, v, out, 128, 128, 0.5)
+    assert e.value.status == sb.SOL_ERR_WORKSPACE
+    # misaligned pointer
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q.view(-1)[1:1 + 256 * 128 - 128].view(1, 1, 255, 128), k, v, out, ws, 128, 128)
+    assert e.value.status in (sb.SOL_ERR_INVALID_ARG, sb.SOL_ERR_WORKSPACE)
+
+
+def test_bound_entry_points_and_host_path():
+    wl = WORKLOADS["tiny"]
+    beta = load_betas()["tiny"][0.3]
+    qb, kb, vb = synth.generate(wl)
+    q, k, v = hp.to_dev(qb), hp.to_dev(kb), hp.to_dev(vb)
+    ws = sb.make_workspace(wl.batch, wl.heads, wl.seq_len, wl.d, wl.block, wl.block)
+    sb.sol_attn_bind_workspace(ws)
+    out = torch.empty_like(q)
+    sb.sol_attn_forward(q, k, v, out, wl.block, wl.block, beta)
+    torch.cuda.synchronize()
+    ref, _, _, _ = hp.run_gpu(q, k, v, wl.block, beta)
+    assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+    # host-buffer entry point
+    hq, hk, hv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (qb, kb, vb))
+    hout = torch.empty_like(hq).pin_memory()
+    dq, dk, dv, dout = (torch.empty_like(q) for _ in range(4))
+    sb.sol_attn_bind_workspace(ws)
+    sb.sol_attn_forward_host(hq, hk, hv, hout, dq, dk, dv, dout, wl.block, wl.block, beta)
+    torch.cuda.synchronize()
+    assert torch.equal(hout, ref.view(torch.int16).cpu())
+    dense = torch.empty_like(q)
+    sb.sol_attn_dense(q, k, v, dense)
+    torch.cuda.synchronize()
+    for h in range(wl.heads):
+        refd = orc.dense_attention(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                                   synth.widen(vb[0, h], np.float64))
+        assert np.abs(hp.dev_to_f64(dense)[0, h] - refd).max() <= hp.MAX_ABS
