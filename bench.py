@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the Sol-Attn fused forward path on synthetic video-DiT-shaped inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload video720] [--density 0.15] [--no-sweep]
+
+One "step" is one pass of the whole hot path (pooling pre-pass, thresholds, fused kernel) over
+one batch (B=1, H=40, N=75600, d=128, block 128 for the default workload).  Prints ONE JSON line.
+
+* value / unit: dense-equivalent TFLOP/s = 4*B*H*N^2*d / time, inputs resident in HBM.
+* ms_per_step: ms per call (pool + fused kernel).
+* e2e: the same metric through ``sol_attn_forward_host`` with pinned HOST buffers, i.e. with
+  the host->device copies of q, k, v and the device->host copy of the output inside the timed
+  region.
+* roofline: the fused kernel alone (``skip_pool``), computed FLOPs (exact pairs actually routed +
+  the approximate outer loop) per launch / CUDA-event time, against the measured bf16 peak.
+* cpu_baseline: the CPU oracle timed on a bounded sample of the same workload.
+* sweep: every density of the workload's threshold sweep plus the dense-mode run.
+
+Under torchrun every rank runs the same workload on its own GPU (heads are independent; there
+is no collective in the operator), timing is max over ranks and ``value`` is the aggregate.
+``--impl reference`` times the CPU oracle (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_24027_b200 import synth  # noqa: E402
+from paper_2607_24027_b200.configs import DENSITY_SWEEP, WORKLOADS, load_betas  # noqa: E402
+
+METRIC = "dense-equivalent attention throughput at 720p (ms/call in ms_per_step)"
+UNIT = "TFLOP/s (dense-equivalent)"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_burst": p["bf16_tflops"], "bf16_sustained": p.get("bf16_tflops_sustained"),
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def dense_flops(wl):
+    return 4.0 * wl.batch * wl.heads * float(wl.seq_len) ** 2 * wl.d
+
+
+def computed_flops(wl, counts_sum, mode_dense=False):
+    """Algorithmic FLOPs of one fused-kernel launch: routed (query block, key block) pairs are
+    4*b*b*d each; the approximate outer loop is a b x Nk x d pair of GEMMs per query block."""
+    b, d, nk = wl.block, wl.d, wl.n_blocks
+    exact = float(counts_sum) * 4.0 * b * b * d
+    if mode_dense:
+        return exact
+    approx = wl.batch * wl.heads * float(nk) * 4.0 * b * nk * d
+    return exact + approx
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = max(mx, float(f[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arm
+def oracle_sample(wl, beta, n_tiles=6, seed=0):
+    """Time the oracle on a bounded sample: routing of head 0 plus `n_tiles` query blocks of it
+    (Algorithm 1).  Returns (seconds per query block incl. its share of routing, description)."""
+    from oracle import sol_attn_oracle as orc
+    qb, kb, vb = synth.generate(wl, heads=slice(0, 1))
+    q, k, v = (synth.widen(x[0], np.float64) for x in (qb, kb, vb))
+    t0 = time.perf_counter()
+    r = orc.routing(q, k, v, wl.block, wl.block, beta)
+    t_route = time.perf_counter() - t0
+    nq = r.mask.shape[0]
+    rng = np.random.default_rng(seed)
+    tiles = sorted(rng.choice(nq, size=min(n_tiles, nq), replace=False).tolist())
+    t0 = time.perf_counter()
+    orc.sol_attn_streaming(q, k, v, r.kc, r.vc, r.tau, wl.block, wl.block, chunk=16, q_tiles=tiles)
+    t_tiles = time.perf_counter() - t0
+    per_tile = t_tiles / len(tiles) + t_route / nq
+    return per_tile, f"head 0: routing of all {nq} query blocks + Algorithm 1 on query blocks {tiles}", \
+        float(r.mask.mean())
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, wl, beta):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total_tiles = wl.batch * wl.heads * wl.n_blocks
+    times = []
+    sample = ""
+    for step in range(args.warmup + args.steps):
+        per_tile, sample, _ = oracle_sample(wl, beta, n_tiles=4, seed=step)
+        if step >= args.warmup:
+            times.append(per_tile * total_tiles)
+    t = float(np.mean(times))
+    val = dense_flops(wl) / t / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{wl.name} density {args.density}", "B": wl.batch, "H": wl.heads,
+                       "N": wl.seq_len, "d": wl.d, "block": wl.block, "beta": beta,
+                       "note": "each step times a bounded sample and extrapolates by query-block count"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="video720", choices=list(WORKLOADS))
+    ap.add_argument("--density", type=float, default=0.15)
+    ap.add_argument("--kernel", default="auto", choices=["auto", "tcgen05", "mma_sync"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--heads", type=int, default=0, help="override the head count (profiling small cases)")
+    args = ap.parse_args()
+
+    wl = WORKLOADS[args.workload]
+    if args.heads:
+        import dataclasses
+        wl = dataclasses.replace(wl, heads=args.heads)
+    betas = load_betas()[args.workload]
+    if args.density not in betas:
+        raise SystemExit(f"density {args.density} not calibrated for {args.workload}: {sorted(betas)}")
+    beta = betas[args.density]
+
+    if args.impl == "reference":
+        run_reference(args, wl, beta)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_24027_b200 import binding as sb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    sb.lib()   # fails loudly when the CUDA library is missing
+
+    impl = {"auto": sb.SOL_IMPL_AUTO, "tcgen05": sb.SOL_IMPL_TCGEN05, "mma_sync": sb.SOL_IMPL_MMA_SYNC}[args.kernel]
+
+    # inputs: generated on the host by the seeded generator, then kept resident in HBM
+    import dataclasses
+    wl_rank = dataclasses.replace(wl, seed=wl.seed + 1000 * rank) if rank else wl
+    qb, kb, vb = synth.generate(wl_rank)
+    to_dev = lambda x: torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16)
+    q, k, v = to_dev(qb), to_dev(kb), to_dev(vb)
+    out = torch.empty_like(q)
+    B, H, N, d = q.shape
+    ws = sb.make_workspace(B, H, N, d, wl.block, wl.block)
+    sb.sol_attn_bind_workspace(ws)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        """ms per step: CUDA events on the launching stream, max over ranks."""
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def check_status():
+        st = sb.sol_attn_read_device_status()
+        if st != sb.SOL_OK:
+            raise SystemExit(f"device status {sb.status_string(st)}")
+
+    def full_step(b=beta):
+        sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl)
+
+    def kernel_only(b=beta):
+        sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl, skip_pool=True)
+
+    def dense_step():
+        sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, mode=sb.SOL_MODE_DENSE, impl=impl)
+
+    def pool_only():
+        sb.sol_attn_pool(q, k, v, wl.block, wl.block, beta)
+
+    dflops = dense_flops(wl)
+    peaks = load_peaks()
+
+    # ---- headline: whole path, inputs resident
+    launches0 = sb.sol_attn_launch_count()
+    with ClockSampler(local) as clk:
+        ms_step = timed(full_step, args.steps, args.warmup)
+    launches = (sb.sol_attn_launch_count() - launches0) * args.steps // (args.steps + args.warmup)
+    check_status()
+    counts_sum = int(ws.counts.sum().item())
+    density = counts_sum / float(B * H * wl.n_blocks * wl.n_blocks)
+
+    # ---- fused kernel alone (workspace already holds the pre-attention results)
+    ms_kernel = timed(kernel_only, args.steps, 1)
+    cflops = computed_flops(wl, counts_sum)
+    achieved = cflops / (ms_kernel * 1e-3) / 1e12
+    ms_pool = timed(pool_only, args.steps, 1)
+    pool_bytes = 3.0 * B * H * N * d * 2 + 3.0 * B * H * wl.n_blocks * d * 4 + 2.0 * B * H * wl.n_blocks * d * 2
+    check_status()
+
+    # ---- end to end with host buffers
+    hq, hk, hv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (qb, kb, vb))
+    hout = torch.empty_like(hq).pin_memory()
+    dq, dk, dv, dout = (torch.empty_like(q) for _ in range(4))
+
+    def e2e_step():
+        sb.sol_attn_forward_host(hq, hk, hv, hout, dq, dk, dv, dout, wl.block, wl.block, beta)
+
+    ms_e2e = timed(e2e_step, max(2, args.steps // 2), 1)
+    check_status()
+    assert torch.equal(hout.view(-1)[:4096], out.view(torch.int16).view(-1)[:4096].cpu()), "host path disagrees"
+    del hq, hk, hv, hout, dq, dk, dv, dout
+
+    # ---- sweep: every calibrated density + dense mode (kernel-only and whole path)
+    sweep = []
+    if not args.no_sweep:
+        ms_dense = timed(dense_step, max(2, args.steps // 3), 1)
+        dense_cf = computed_flops(wl, B * H * wl.n_blocks * wl.n_blocks, mode_dense=True)
+        sweep.append({"mode": "dense", "ms_per_call": ms_dense, "dense_equiv_tflops": dflops / ms_dense / 1e9,
+                      "frac_of_peak_computed": dense_cf / ms_dense / 1e9 / peaks["bf16_burst"]})
+        for rho in DENSITY_SWEEP[args.workload]:
+            b = betas[rho]
+            ms_f = timed(lambda: full_step(b), max(3, args.steps // 2), 1)
+            cs = int(ws.counts.sum().item())
+            ms_k = timed(lambda: kernel_only(b), max(3, args.steps // 2), 1)
+            dens = cs / float(B * H * wl.n_blocks * wl.n_blocks)
+            cf = computed_flops(wl, cs)
+            sweep.append({"mode": "sol", "target_density": rho, "beta": b, "density": dens,
+                          "ms_per_call": ms_f, "kernel_ms": ms_k, "dense_equiv_tflops": dflops / ms_f / 1e9,
+                          "computed_tflops": cf / ms_k / 1e9,
+                          "frac_of_peak_computed": cf / ms_k / 1e9 / peaks["bf16_burst"],
+                          "speedup_vs_dense": ms_dense / ms_f, "one_over_density": 1.0 / dens})
+        check_status()
+
+    if world > 1:
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only)
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        per_tile, sample, _ = oracle_sample(wl, beta, n_tiles=6)
+        t_cpu = per_tile * B * H * wl.n_blocks
+        cpu = {"value": dflops / t_cpu / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": sample + f"; {per_tile:.3f} s per query block, extrapolated x{B * H * wl.n_blocks}"}
+
+    line = {
+        "metric": METRIC, "value": world * dflops / (ms_step * 1e-3) / 1e12, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{wl.name} density {args.density}", "B": B, "H": H, "N": N, "d": d,
+                   "block": wl.block, "beta": beta, "achieved_density": density, "kernel": args.kernel,
+                   "l2": "inputs (3 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
+                   "parallelism": "replicas (no collective)" if world > 1 else "single GPU"},
+        "clocks": clk.summary(),
+        "e2e": {"value": world * dflops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": q.numel() * 2},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "fwd_sm100_kernel" if args.kernel != "mma_sync" else "fwd_mma_sync_kernel",
+                     "achieved": achieved, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
+                     "frac": achieved / peaks["bf16_burst"], "peak_source": peaks["source"] + " burst",
+                     "frac_of_sustained": (achieved / peaks["bf16_sustained"]) if peaks["bf16_sustained"] else None,
+                     "kernel_ms": ms_kernel, "computed_flops": cflops, "traffic": None},
+        "pool": {"bound": "hbm", "ms": ms_pool, "achieved": pool_bytes / (ms_pool * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                 "unit": "GB/s", "frac": pool_bytes / (ms_pool * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                 "note": "pool + moments + tau kernels together"},
+        "cpu_baseline": cpu,
+        "sweep": sweep,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

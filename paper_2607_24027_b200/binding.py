@@ -14,7 +14,7 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libsol_attn.so")
+LIB_PATH = os.environ.get("SOL_ATTN_LIB", os.path.join(_PKG, "libsol_attn.so"))   # override: profiling build
 
 SOL_OK = 0
 SOL_ERR_INVALID_ARG = -1

@@ -32,18 +32,29 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every kernel for sm_100a and link the C-ABI library; returns its path."""
+def build(force: bool = False, verbose: bool = False, profile: bool = False) -> str:
+    """Compile every kernel for sm_100a and link the C-ABI library; returns its path.
+
+    ``profile=True`` builds ``libsol_attn_prof.so`` instead, whose fused kernel records how many
+    cycles each warp role spends in each kind of wait (a development aid, never the default).
+    """
+    if profile:
+        return _build_variant(os.path.join(PKG, "libsol_attn_prof.so"), ["-DSOL_PROFILE"], "_prof", verbose)
     if not force and not _stale():
         return LIB
+    return _build_variant(LIB, [], "", verbose)
+
+
+def _build_variant(lib: str, defines, suffix: str, verbose: bool) -> str:
     objs = []
     common = [_nvcc(), "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    common += defines
     if verbose:
         common += ["-Xptxas", "-v"]
     procs = []
     for s in SOURCES:
-        obj = os.path.join(CSRC, s.replace(".cu", ".o"))
+        obj = os.path.join(CSRC, s.replace(".cu", suffix + ".o"))
         objs.append(obj)
         procs.append((s, subprocess.Popen(common + ["-c", os.path.join(CSRC, s), "-o", obj],
                                           stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -55,11 +66,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", LIB] + objs + ["-lcudart"]
+    link = [_nvcc(), "-shared", "-o", lib] + objs + ["-lcudart"]
     subprocess.run(link, check=True)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv)
+    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, profile="--profile" in sys.argv)
     print(path)

@@ -40,6 +40,8 @@ constexpr int kStages = 2;                      // ring of K/V tiles
 constexpr int kRecords = 4;                     // ring of routing records
 constexpr int kTmemCols = 256;                  // S: [0,128)  O: [128,256);  P (bf16) aliases S [0,64)
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
+constexpr int kPolyEvery = 4;                   // every 4th exp2 runs on the FMA pipe (0: none)
+constexpr int kSoftmaxRegs = 184, kOtherRegs = 72;   // setmaxnreg split of the 2 x 128 x 128 budget
 
 constexpr uint8_t kRecFirst = 1, kRecLast = 2, kRecApprox = 4;
 
@@ -80,8 +82,56 @@ __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int wher
   atomicExch(p.status + kStatusDetail, where);
 }
 
-#define SOL_WAIT(bar, parity, where)                                  \
-  if (!mbar_wait((bar), (parity), &sm.abort_flag)) {                  \
+// 2^x for x <= ~8 without the MUFU unit: round-to-nearest split x = n + f, f in [-0.5, 0.5],
+// cubic minimax polynomial for 2^f (max relative error 7.5e-5, far below bf16 resolution), and n
+// added straight into the exponent field.
+__device__ __forceinline__ float exp2_poly(float x) {
+  x = fmaxf(x, -126.f);
+  const float magic = 12582912.f;               // 1.5 * 2^23: the low mantissa bits of x + magic hold n
+  const float r = x + magic;
+  const float f = x - (r - magic);
+  const float pz = fmaf(fmaf(fmaf(0.055171460f, f, 0.24261086f), f, 0.69326097f), f, 0.99992812f);
+  return __int_as_float(__float_as_int(pz) + (__float_as_int(r) << 23));
+}
+
+// Optional per-role cycle accounting (build with -DSOL_PROFILE): how long each role spends in
+// each kind of wait.  Slot meaning is listed next to every use; read back with
+// sol_attn_debug_profile().
+#ifdef SOL_PROFILE
+constexpr int kProfCtas = 512, kProfRoles = 4, kProfSlots = 8;
+__device__ long long g_prof[kProfCtas * kProfRoles * kProfSlots];
+struct Prof {
+  long long v[kProfSlots];
+  long long t0;
+  __device__ Prof() {
+    for (int i = 0; i < kProfSlots; ++i) v[i] = 0;
+    t0 = clock64();
+  }
+  __device__ void flush(int role) {
+    v[kProfSlots - 1] = clock64() - t0;
+    if (blockIdx.x < kProfCtas)
+      for (int i = 0; i < kProfSlots; ++i) g_prof[(blockIdx.x * kProfRoles + role) * kProfSlots + i] = v[i];
+  }
+};
+__device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long& acc) {
+  const long long t = clock64();
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  acc += clock64() - t;
+  return ok;
+}
+#define WAIT(bar, parity, slot) prof_wait((bar), (parity), &sm.abort_flag, prof.v[slot])
+#define PROF_DECL Prof prof;
+#define PROF_COUNT(slot) (++prof.v[slot])
+#define PROF_FLUSH(role) prof.flush(role)
+#else
+#define WAIT(bar, parity, slot) mbar_wait((bar), (parity), &sm.abort_flag)
+#define PROF_DECL
+#define PROF_COUNT(slot)
+#define PROF_FLUSH(role)
+#endif
+
+#define SOL_WAIT(bar, parity, where, slot)                            \
+  if (!WAIT((bar), (parity), (slot))) {                               \
     flag_abort(sm, p, (where));                                       \
     break;                                                            \
   }
@@ -89,6 +139,7 @@ __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int wher
 // ------------------------------------------------------------------------------------------------
 // router: one warp
 __device__ void router_role(Shared& sm, const Params& p, int lane) {
+  PROF_DECL
   const unsigned full = 0xffffffffu;
   uint32_t n_rec = 0;
   const int n_chunks = ceil_div(p.Nk, kBlk);
@@ -110,7 +161,7 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
     int count = 0;
     for (int t = 0; t < n_chunks; ++t) {
       Record& rec = sm.rec[n_rec % kRecords];
-      if (!mbar_wait(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, &sm.abort_flag)) {
+      if (!WAIT(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, 0)) {   // prof 0: record ring full
         if (lane == 0) flag_abort(sm, p, 100);
         alive = false;
         break;
@@ -128,24 +179,34 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
         } else {
           // partial dot products of 32 pooled keys (lane owns channels 4*lane..4*lane+3), then a
           // transposing butterfly leaves the full dot product of key jbase+l in lane l
-          float v[32];
+          // lane owns channels 4*lane..4*lane+3.  Eight pooled keys at a time: partial dot
+          // products, a transposing butterfly over lane bits 0-2 and two plain exchanges leave the
+          // dot product of key (8*sub + (lane & 7)) in every lane; lanes 8*sub..8*sub+7 keep it.
+          float dot = 0.f;
+#pragma unroll 1
+          for (int sub = 0; sub < 4; ++sub) {
+            float v[8];
 #pragma unroll
-          for (int r = 0; r < 32; ++r) {
-            const int jr = min(jbase + r, p.Nk - 1);
-            const float4 kk = __ldg(reinterpret_cast<const float4*>(kc_head + (size_t)jr * kD + lane * 4));
-            v[r] = fmaf(qb.x, kk.x, fmaf(qb.y, kk.y, fmaf(qb.z, kk.z, qb.w * kk.w)));
-          }
-#pragma unroll
-          for (int off = 16; off >= 1; off >>= 1) {
-#pragma unroll
-            for (int r = 0; r < off; ++r) {
-              const bool up = (lane & off) != 0;
-              const float send = up ? v[r] : v[r + off];
-              const float keep = up ? v[r + off] : v[r];
-              v[r] = keep + __shfl_xor_sync(full, send, off);
+            for (int r = 0; r < 8; ++r) {
+              const int jr = min(jbase + sub * 8 + r, p.Nk - 1);
+              const float4 kk = __ldg(reinterpret_cast<const float4*>(kc_head + (size_t)jr * kD + lane * 4));
+              v[r] = fmaf(qb.x, kk.x, fmaf(qb.y, kk.y, fmaf(qb.z, kk.z, qb.w * kk.w)));
             }
+#pragma unroll
+            for (int off = 4; off >= 1; off >>= 1) {
+#pragma unroll
+              for (int r = 0; r < off; ++r) {
+                const bool up = (lane & off) != 0;
+                const float send = up ? v[r] : v[r + off];
+                const float keep = up ? v[r + off] : v[r];
+                v[r] = keep + __shfl_xor_sync(full, send, off);
+              }
+            }
+            v[0] += __shfl_xor_sync(full, v[0], 8);
+            v[0] += __shfl_xor_sync(full, v[0], 16);
+            if ((lane >> 3) == sub) dot = v[0];
           }
-          sel = (j < p.Nk) && (p.scale * v[0] > tau_i);
+          sel = (j < p.Nk) && (p.scale * dot > tau_i);
         }
         const unsigned m = __ballot_sync(full, sel);
         const bool valid = j < p.Nk;
@@ -170,6 +231,7 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
     }
     if (alive && lane == 0 && p.counts) p.counts[w] = count;
   }
+  PROF_FLUSH(0);
   // end-of-stream record
   if (alive) {
     if (mbar_wait(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, &sm.abort_flag)) {
@@ -189,9 +251,10 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
                               const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vm) {
   uint32_t n_rec = 0, n_load = 0, n_item = 0;
+  PROF_DECL
   auto load_tile = [&](const CUtensorMap* tm, int row, int bh) -> bool {
     const uint32_t s = n_load % kStages;
-    if (!mbar_wait(&sm.kv_empty[s], ((n_load / kStages) & 1) ^ 1, &sm.abort_flag)) return false;
+    if (!WAIT(&sm.kv_empty[s], ((n_load / kStages) & 1) ^ 1, 1)) return false;   // prof 1: K/V ring full
     mbar_arrive_expect_tx(&sm.kv_full[s], kTileBytes);
     unsigned char* dst = sKV + (size_t)s * kTileBytes;
     tma_load_3d(dst, tm, &sm.kv_full[s], 0, row, bh);
@@ -201,7 +264,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
   };
   for (;;) {
     const uint32_t r = n_rec % kRecords;
-    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 200);
+    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 200, 0);                   // prof 0: no record yet
     const Record& rec = sm.rec[r];
     const int w = rec.work;
     if (w < 0) break;
@@ -209,7 +272,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     const int j0 = rec.chunk * kBlk;
     bool ok = true;
     if (rec.flags & kRecFirst) {
-      SOL_WAIT(&sm.q_empty, (n_item & 1) ^ 1, 201);
+      SOL_WAIT(&sm.q_empty, (n_item & 1) ^ 1, 201, 2);                         // prof 2: Q slot busy
       mbar_arrive_expect_tx(&sm.q_full, kTileBytes);
       tma_load_3d(sQ, tm_q, &sm.q_full, 0, i * kBlk, bh);
       tma_load_3d(sQ + kHalfBytes, tm_q, &sm.q_full, 64, i * kBlk, bh);
@@ -225,6 +288,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     mbar_arrive(&sm.rec_empty[r]);
     ++n_rec;
   }
+  PROF_FLUSH(1);
   if (sm.abort_flag) {
     // let copies that are still in flight land before the CTA's shared memory goes away
     int never = 0;                                   // this drain must not be cut short by the abort flag
@@ -244,9 +308,10 @@ __device__ void mma_role(Shared& sm, const Params& p, unsigned char* sQ, unsigne
   const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
   uint32_t n_rec = 0, n_load = 0, n_item = 0, g = 0;   // g: tiles issued so far by this CTA
   int tiles_in_item = 0;
+  PROF_DECL
   for (;;) {
     const uint32_t r = n_rec % kRecords;
-    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 300);
+    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 300, 0);                   // prof 0: no record yet
     const Record& rec = sm.rec[r];
     if (rec.work < 0) break;
     const uint8_t flags = rec.flags;
@@ -255,16 +320,16 @@ __device__ void mma_role(Shared& sm, const Params& p, unsigned char* sQ, unsigne
     ++n_rec;
     bool ok = true;
     if (flags & kRecFirst) {
-      if (!mbar_wait(&sm.q_full, n_item & 1, &sm.abort_flag)) { flag_abort(sm, p, 301); break; }
+      if (!WAIT(&sm.q_full, n_item & 1, 1)) { flag_abort(sm, p, 301); break; }      // prof 1: Q not loaded
       ++n_item;
       tiles_in_item = 0;
     }
     for (int e = 0; e < n_tiles; ++e) {
       // ---- S = Q K^T
       const uint32_t sk = n_load % kStages;
-      if (!mbar_wait(&sm.kv_full[sk], (n_load / kStages) & 1, &sm.abort_flag)) { ok = false; break; }
+      if (!WAIT(&sm.kv_full[sk], (n_load / kStages) & 1, 2)) { ok = false; break; }   // prof 2: K not loaded
       ++n_load;
-      if (g > 0 && !mbar_wait(&sm.pv_done, (g - 1) & 1, &sm.abort_flag)) { ok = false; break; }   // P of the previous tile consumed
+      if (g > 0 && !WAIT(&sm.pv_done, (g - 1) & 1, 3)) { ok = false; break; }         // prof 3: previous P V still running
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
@@ -276,9 +341,9 @@ __device__ void mma_role(Shared& sm, const Params& p, unsigned char* sQ, unsigne
       mma_commit(&sm.s_full);
       // ---- O += P V
       const uint32_t sv = n_load % kStages;
-      if (!mbar_wait(&sm.kv_full[sv], (n_load / kStages) & 1, &sm.abort_flag)) { ok = false; break; }
+      if (!WAIT(&sm.kv_full[sv], (n_load / kStages) & 1, 4)) { ok = false; break; }   // prof 4: V not loaded
       ++n_load;
-      if (!mbar_wait(&sm.p_full, g & 1, &sm.abort_flag)) { ok = false; break; }
+      if (!WAIT(&sm.p_full, g & 1, 5)) { ok = false; break; }                         // prof 5: softmax not done
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < kBlk / 16; ++ks) {
@@ -293,6 +358,7 @@ __device__ void mma_role(Shared& sm, const Params& p, unsigned char* sQ, unsigne
     if (!ok) { flag_abort(sm, p, 302); break; }
     if (flags & kRecLast) mma_commit(&sm.q_empty);     // every MMA that reads Q_i has been issued
   }
+  PROF_FLUSH(2);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -303,13 +369,15 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
   const uint32_t t_s = lane_base, t_o = lane_base + 128;
   const int row = warp * 32 + lane;
   const float sl2 = p.scale * 1.4426950408889634f;
+  const float inv_sl2 = 1.f / sl2;
   uint32_t n_rec = 0, g = 0;
   int tiles_in_item = 0;
   float m_used = 0.f, l = 0.f;
   bool alive = true;
+  PROF_DECL
   while (alive) {
     const uint32_t r = n_rec % kRecords;
-    if (!mbar_wait(&sm.rec_full[r], (n_rec / kRecords) & 1, &sm.abort_flag)) { flag_abort(sm, p, 400); break; }
+    if (!WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 0)) { flag_abort(sm, p, 400); break; }   // prof 0: no record yet
     const Record& rec = sm.rec[r];
     const int w = rec.work;
     if (w < 0) break;
@@ -326,30 +394,34 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
         cols_valid = min(kBlk, p.N - j * kBlk);
       }
       const bool general = approx || cols_valid < kBlk;
-      if (!mbar_wait(&sm.s_full, g & 1, &sm.abort_flag)) { flag_abort(sm, p, 401); alive = false; break; }
+      if (!WAIT(&sm.s_full, g & 1, 1)) { flag_abort(sm, p, 401); alive = false; break; }   // prof 1: S not ready
       tc_fence_after();
-      // ---- pass 1: row maximum (log2 domain)
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-        uint32_t a[32], b[32];
-        tmem_ld_32x32b_x32(t_s + h * 64, a);
-        tmem_ld_32x32b_x32(t_s + h * 64 + 32, b);
-        tmem_ld_wait();
-        if (!general) {
+      // ---- the whole row of S (128 fp32) into registers with one wait
+      uint32_t sr[kBlk];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) mx = fmaxf(mx, fmaxf(__uint_as_float(a[c]), __uint_as_float(b[c])));
-        } else {
+      for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+      tmem_ld_wait();
+      if (general) {
+        // bring the rare tiles (approximate chunk, ragged last block) to the common form
+        // logit = sl2 * x by folding the column bias into x; -inf marks masked columns
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int c0 = h * 64 + c, c1 = c0 + 32;
-            const float b0 = approx ? rec.bias[c0] : (c0 < cols_valid ? 0.f : -INFINITY);
-            const float b1 = approx ? rec.bias[c1] : (c1 < cols_valid ? 0.f : -INFINITY);
-            mx = fmaxf(mx, fmaxf(fmaf(__uint_as_float(a[c]), sl2, b0), fmaf(__uint_as_float(b[c]), sl2, b1)));
-          }
+        for (int c = 0; c < kBlk; ++c) {
+          const float x = __uint_as_float(sr[c]);
+          sr[c] = __float_as_uint(approx ? fmaf(rec.bias[c], inv_sl2, x) : (c < cols_valid ? x : -INFINITY));
         }
       }
-      if (!general) mx *= sl2;
+      float mx;
+      {
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          m0 = fmaxf(m0, __uint_as_float(sr[c]));
+          m1 = fmaxf(m1, __uint_as_float(sr[32 + c]));
+          m2 = fmaxf(m2, __uint_as_float(sr[64 + c]));
+          m3 = fmaxf(m3, __uint_as_float(sr[96 + c]));
+        }
+        mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sl2;
+      }
       // ---- running maximum, lazy rescale of O
       if (tiles_in_item == 0) {
         m_used = mx;
@@ -357,7 +429,8 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
       } else if (__any_sync(full, mx > m_used + kRescaleThreshold)) {
         const float m_new = fmaxf(m_used, mx);
         const float f = ex2(m_used - m_new);
-        if (!mbar_wait(&sm.pv_done, (g - 1) & 1, &sm.abort_flag)) { flag_abort(sm, p, 402); alive = false; break; }
+        PROF_COUNT(4);                                                                   // prof 4: number of rescales
+        if (!WAIT(&sm.pv_done, (g - 1) & 1, 2)) { flag_abort(sm, p, 402); alive = false; break; }
         tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -371,49 +444,33 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
         l *= f;
         m_used = m_new;
       }
-      // ---- pass 2: P = exp2(S - m), row sum, P (bf16) back to TMEM over S
-#pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-        uint32_t a[32], b[32];
-        tmem_ld_32x32b_x32(t_s + h * 64, a);
-        tmem_ld_32x32b_x32(t_s + h * 64 + 32, b);
-        tmem_ld_wait();
-        float sum0 = 0.f, sum1 = 0.f;
-        if (!general) {
-          const float nm = -m_used;
+      // ---- P = exp2(sl2 * S - m): most elements on the MUFU unit, every kPolyEvery-th one as a
+      //      polynomial on the FMA pipe; row sum; P (bf16) back to TMEM over the first half of S
+      {
+        const float nm = -m_used;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float pa = ex2(fmaf(__uint_as_float(a[c]), sl2, nm));
-            const float pb = ex2(fmaf(__uint_as_float(b[c]), sl2, nm));
-            sum0 += pa; sum1 += pb;
-            a[c] = __float_as_uint(pa); b[c] = __float_as_uint(pb);
+        for (int c = 0; c < kBlk; c += 4) {
+          float e[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float x = fmaf(__uint_as_float(sr[c + u]), sl2, nm);
+            e[u] = (kPolyEvery > 0 && ((c + u) % kPolyEvery) == kPolyEvery - 1) ? exp2_poly(x) : ex2(x);
           }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int c0 = h * 64 + c, c1 = c0 + 32;
-            const float b0 = approx ? rec.bias[c0] : (c0 < cols_valid ? 0.f : -INFINITY);
-            const float b1 = approx ? rec.bias[c1] : (c1 < cols_valid ? 0.f : -INFINITY);
-            const float pa = ex2(fmaf(__uint_as_float(a[c]), sl2, b0 - m_used));
-            const float pb = ex2(fmaf(__uint_as_float(b[c]), sl2, b1 - m_used));
-            sum0 += pa; sum1 += pb;
-            a[c] = __float_as_uint(pa); b[c] = __float_as_uint(pb);
-          }
+          sum0 += e[0]; sum1 += e[1]; sum2 += e[2]; sum3 += e[3];
+          __nv_bfloat162 lo = __floats2bfloat162_rn(e[0], e[1]);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(e[2], e[3]);
+          sr[c / 2] = *reinterpret_cast<uint32_t*>(&lo);
+          sr[c / 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
         }
-        l += sum0 + sum1;
-        uint32_t pk[32];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          __nv_bfloat162 x = __floats2bfloat162_rn(__uint_as_float(a[2 * c]), __uint_as_float(a[2 * c + 1]));
-          __nv_bfloat162 y = __floats2bfloat162_rn(__uint_as_float(b[2 * c]), __uint_as_float(b[2 * c + 1]));
-          pk[c] = *reinterpret_cast<uint32_t*>(&x);
-          pk[16 + c] = *reinterpret_cast<uint32_t*>(&y);
-        }
-        tmem_st_32x32b_x32(t_s + h * 32, pk);
+        l += (sum0 + sum1) + (sum2 + sum3);
+        tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+        tmem_st_32x32b_x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       }
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&sm.p_full);
+      PROF_COUNT(5);                                                                     // prof 5: tiles
       ++g;
       ++tiles_in_item;
     }
@@ -424,7 +481,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
       const int q_rows = min(kBlk, p.N - i * kBlk);
       __nv_bfloat16* orow = p.out + ((size_t)bh * p.N + (size_t)i * kBlk + row) * kD;
       if (tiles_in_item > 0) {
-        if (!mbar_wait(&sm.pv_done, (g - 1) & 1, &sm.abort_flag)) { flag_abort(sm, p, 403); break; }
+        if (!WAIT(&sm.pv_done, (g - 1) & 1, 3)) { flag_abort(sm, p, 403); break; }           // prof 3: last P V of the item
         tc_fence_after();
         const float inv = 1.f / l;
 #pragma unroll 1
@@ -458,6 +515,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
     if (lane == 0) mbar_arrive(&sm.rec_empty[r]);
     ++n_rec;
   }
+  if (lane == 0 && warp == 0) PROF_FLUSH(3);
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -490,8 +548,12 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem = sm.tmem_base;
 
   if (warp < 4) {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     softmax_role(sm, p, tmem, warp, lane);
-  } else if (warp == 4) {
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+  }
+  if (warp == 4) {
     router_role(sm, p, lane);
   } else if (warp == 5) {
     if (lane == 0) producer_role(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
@@ -504,6 +566,17 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 }
 
 }  // namespace
+
+#ifdef SOL_PROFILE
+}  // namespace sol
+// Debug builds only: copies the per-CTA, per-role wait-cycle counters of the last launch to the host.
+extern "C" int sol_attn_debug_profile(long long* host_out, int n_values) {
+  const size_t total = sizeof(long long) * sol::kProfCtas * sol::kProfRoles * sol::kProfSlots;
+  const size_t want = sizeof(long long) * (size_t)n_values;
+  return (int)cudaMemcpyFromSymbol(host_out, sol::g_prof, want < total ? want : total);
+}
+namespace sol {
+#endif
 
 bool fwd_sm100_supports(const Problem& p) { return p.d == kD && p.block_q == kBlk && p.block_k == kBlk; }
 
