@@ -1,24 +1,31 @@
 // Sol-Attn fused forward (Algorithm 1) for sm_100a: TMA + tcgen05.mma + TMEM.
 //
-// Persistent kernel, two CTAs per SM, d = 128, block_q = block_k = 128.  A CTA owns one query
-// block at a time and is split into warp roles that talk through mbarriers:
+// Persistent kernel, one CTA of 384 threads per SM, d = 128, block_q = block_k = 128.  A CTA owns
+// one query block at a time and is split into warp roles that talk through mbarriers:
 //
-//   router   (warp 4)  pulls (head, query block) work items from a global counter and walks the
+//   router   (warp 8)  pulls (head, query block) work items from a global counter and walks the
 //                      pooled keys in chunks of 128 blocks.  For every block it evaluates the
 //                      proxy s_ij = scale * Qbar_i . KC_j (Eq. 3) in fp32 and compares it with
 //                      tau_i (Eq. 4).  The decision only ever lives in a small shared-memory
 //                      record (selected list + per-column bias); nothing of the proxy map goes
 //                      to global memory.
-//   producer (warp 5)  reads the records and issues TMA loads: one approximate tile per chunk
+//   producer (warp 9)  reads the records and issues TMA loads: one approximate tile per chunk
 //                      (KC chunk, mean-V chunk) and K_j / V_j ONLY for routed blocks.
-//   mma      (warp 6)  one thread issues tcgen05.mma: S = Q K^T into TMEM, then O += P V with P
-//                      read from TMEM (where the softmax warps left it) and V from shared memory.
-//   softmax  (warps 0-3, one thread per query row) online softmax over the tile stream; both
-//                      branches update the same (m, l, O): an approximate tile is an ordinary
-//                      tile whose columns carry the bias log2(n_j) (Eqs. 9-10: multiplicity n_j
-//                      in the denominator, mean value times n_j in the numerator) or -inf for
-//                      routed / padded columns.  O is rescaled lazily, only when the running
-//                      maximum grows by more than 2^8.
+//   mma      (warps 10, 11) one thread each issues tcgen05.mma: warp 10 the score GEMMs S = Q K^T,
+//                      warp 11 the value GEMMs O += P V.  S goes to one of two TMEM score buffers,
+//                      so the scores of tile g+1 are computed while tile g is in softmax.
+//   softmax  (warps 0-3 and 4-7) two warpgroups; thread = query row; group h owns key columns
+//                      [64h, 64h+64) of EVERY tile and keeps its own running (m_h, l_h) and its own
+//                      accumulator O_h in TMEM (O_h += P_h V[64h:64h+64]); the two partial results
+//                      are merged when the query block is finished.  Both branches of the method
+//                      update the same state: an approximate tile is an ordinary tile whose
+//                      columns carry the bias log2(n_j) (Eqs. 9-10: multiplicity n_j in the
+//                      denominator, mean value times n_j in the numerator) or -inf for routed /
+//                      padded columns.  O_h is rescaled lazily, only when the running maximum
+//                      grows by more than 2^8.
+//
+// TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512); P_h (bf16) of a tile
+// overwrites the first 32 columns of group h's half of that tile's S buffer.
 //
 // Every mbarrier wait is bounded: when one expires the CTA records SOL_ERR_DEVICE_TIMEOUT in the
 // workspace status word, all roles drain, TMEM is released and the kernel returns.
@@ -33,15 +40,17 @@ using namespace ptx;
 
 constexpr int kD = 128;
 constexpr int kBlk = 128;
-constexpr int kThreads = 256;
-constexpr int kTileBytes = kBlk * kD * 2;       // 32 KB: one K-like or V-like tile
-constexpr int kHalfBytes = kTileBytes / 2;      // 16 KB: 64 channels x 128 rows (one TMA box)
-constexpr int kStages = 2;                      // ring of K/V tiles
-constexpr int kRecords = 4;                     // ring of routing records
-constexpr int kTmemCols = 256;                  // S: [0,128)  O: [128,256);  P (bf16) aliases S [0,64)
-constexpr float kRescaleThreshold = 8.0f;       // log2 units
-constexpr int kPolyEvery = 4;                   // every 4th exp2 runs on the FMA pipe (0: none)
-constexpr int kSoftmaxRegs = 184, kOtherRegs = 72;   // setmaxnreg split of the 2 x 128 x 128 budget
+constexpr int kHalf = 64;                        // key columns per softmax warpgroup
+constexpr int kThreads = 384;
+constexpr int kTileBytes = kBlk * kD * 2;        // 32 KB: one K-like or V-like tile
+constexpr int kHalfBytes = kTileBytes / 2;       // 16 KB: 64 channels x 128 rows (one TMA box)
+constexpr int kStages = 5;                       // ring of K/V tiles
+constexpr int kRecords = 4;                      // ring of routing records
+constexpr int kTmemCols = 512;
+constexpr int kTmemS = 0, kTmemO = 256;
+constexpr float kRescaleThreshold = 8.0f;        // log2 units
+constexpr int kStaggerCycles = 500;              // head start of softmax group 0 over group 1, per work item
+constexpr int kPolyEvery = 0;                    // every n-th exp2 runs on the FMA pipe instead of MUFU (0: none)
 
 constexpr uint8_t kRecFirst = 1, kRecLast = 2, kRecApprox = 4;
 
@@ -56,10 +65,12 @@ struct Record {
 
 struct Shared {
   Record rec[kRecords];
+  float2 ml[2][kBlk];           // (m_h, l_h) exchange between the softmax warpgroups
   uint64_t rec_full[kRecords], rec_empty[kRecords];
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t q_full, q_empty;
-  uint64_t s_full, p_full, pv_done;
+  uint64_t s_full[2], p_full[2][2], pv_done[2];   // indexed by score buffer (and warpgroup)
+  uint64_t x_full, x_done;      // rendezvous of the two softmax warpgroups at the end of a work item
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -98,7 +109,7 @@ __device__ __forceinline__ float exp2_poly(float x) {
 // each kind of wait.  Slot meaning is listed next to every use; read back with
 // sol_attn_debug_profile().
 #ifdef SOL_PROFILE
-constexpr int kProfCtas = 512, kProfRoles = 4, kProfSlots = 8;
+constexpr int kProfCtas = 512, kProfRoles = 4, kProfSlots = 12;
 __device__ long long g_prof[kProfCtas * kProfRoles * kProfSlots];
 struct Prof {
   long long v[kProfSlots];
@@ -123,28 +134,107 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_DECL Prof prof;
 #define PROF_COUNT(slot) (++prof.v[slot])
 #define PROF_FLUSH(role) prof.flush(role)
+#define PROF_ACC(slot) (&prof.v[slot])
+#define PROF_T0 const long long prof_t0 = clock64();
+#define PROF_ADD(slot) prof.v[slot] += clock64() - prof_t0;
 #else
 #define WAIT(bar, parity, slot) mbar_wait((bar), (parity), &sm.abort_flag)
 #define PROF_DECL
 #define PROF_COUNT(slot)
 #define PROF_FLUSH(role)
+#define PROF_ACC(slot) nullptr
+#define PROF_T0
+#define PROF_ADD(slot)
 #endif
 
-#define SOL_WAIT(bar, parity, where, slot)                            \
-  if (!WAIT((bar), (parity), (slot))) {                               \
-    flag_abort(sm, p, (where));                                       \
-    break;                                                            \
+// ------------------------------------------------------------------------------------------------
+// Walks the record ring and turns it into a flat stream of events: one per tile, one at the end of
+// every work item, one at the end of the stream.  The producer, the MMA thread and both softmax
+// warpgroups each run their own cursor over the same records.
+enum : int { kEvTile = 0, kEvItemEnd = 1, kEvEnd = 2, kEvAbort = 3 };
+struct Event {
+  int type;
+  int work;          // bh * Nq + i
+  int block;         // tile: key block index j (exact) or first block of the chunk (approximate)
+  bool approx;       // tile: approximate-branch tile
+  bool first;        // tile: first tile of its work item; item end: the item had no tile at all
+  const Record* rec; // tile: its record (bias of an approximate tile)
+};
+
+struct Cursor {
+  uint32_t n_rec = 0;
+  int e = 0;                 // next tile of the current record
+  int n_tiles = 0;
+  int work = 0;              // fields of the open record, cached in registers
+  int block0 = 0;
+  bool has_approx = false;
+  bool have = false;         // a record is open
+  bool item_has_tiles = false;
+  bool end_pending = false;
+  const Record* rec = nullptr;
+};
+
+// `release` is called when the cursor is done with a record (arrives on rec_empty as appropriate
+// for the role).  Returns kEvAbort when a bounded wait expired.
+template <class Release>
+__device__ __forceinline__ Event next_event(Shared& sm, Cursor& c, long long* wait_acc, Release release) {
+  Event ev{};
+  for (;;) {
+    if (!c.have) {
+      const uint32_t r = c.n_rec % kRecords;
+#ifdef SOL_PROFILE
+      const long long t = clock64();
+#endif
+      const bool ok = mbar_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1, &sm.abort_flag);
+#ifdef SOL_PROFILE
+      if (wait_acc) *wait_acc += clock64() - t;
+#endif
+      if (!ok) { ev.type = kEvAbort; return ev; }
+      c.rec = &sm.rec[r];
+      c.work = c.rec->work;
+      if (c.work < 0) { ev.type = kEvEnd; return ev; }
+      const uint32_t flags = c.rec->flags;
+      c.have = true;
+      c.e = 0;
+      c.has_approx = (flags & kRecApprox) != 0;
+      c.n_tiles = (c.has_approx ? 1 : 0) + c.rec->n_sel;
+      c.block0 = c.rec->chunk * kBlk;
+      if (flags & kRecFirst) c.item_has_tiles = false;
+      c.end_pending = (flags & kRecLast) != 0;
+    }
+    if (c.e < c.n_tiles) {
+      ev.type = kEvTile;
+      ev.work = c.work;
+      ev.approx = c.has_approx && c.e == 0;
+      ev.block = c.block0 + (ev.approx ? 0 : c.rec->sel[c.e - (c.has_approx ? 1 : 0)]);
+      ev.first = !c.item_has_tiles;
+      ev.rec = c.rec;
+      c.item_has_tiles = true;
+      ++c.e;
+      return ev;
+    }
+    if (c.end_pending) {
+      c.end_pending = false;
+      ev.type = kEvItemEnd;
+      ev.work = c.work;
+      ev.first = !c.item_has_tiles;
+      return ev;
+    }
+    release(c.n_rec % kRecords);
+    c.have = false;
+    ++c.n_rec;
   }
+}
 
 // ------------------------------------------------------------------------------------------------
 // router: one warp
 __device__ void router_role(Shared& sm, const Params& p, int lane) {
-  PROF_DECL
   const unsigned full = 0xffffffffu;
   uint32_t n_rec = 0;
   const int n_chunks = ceil_div(p.Nk, kBlk);
   const int mask_words = ceil_div(p.Nk, 32);
   bool alive = true;
+  PROF_DECL
   while (alive) {
     int w = 0;
     if (lane == 0) w = atomicAdd(p.status + kStatusTileCounter, 1);
@@ -177,8 +267,6 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
         if (p.mode == SOL_MODE_DENSE) {
           sel = j < p.Nk;
         } else {
-          // partial dot products of 32 pooled keys (lane owns channels 4*lane..4*lane+3), then a
-          // transposing butterfly leaves the full dot product of key jbase+l in lane l
           // lane owns channels 4*lane..4*lane+3.  Eight pooled keys at a time: partial dot
           // products, a transposing butterfly over lane bits 0-2 and two plain exchanges leave the
           // dot product of key (8*sub + (lane & 7)) in every lane; lanes 8*sub..8*sub+7 keep it.
@@ -250,7 +338,8 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
 __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV,
                               const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vm) {
-  uint32_t n_rec = 0, n_load = 0, n_item = 0;
+  uint32_t n_load = 0, n_item = 0;
+  Cursor cur;
   PROF_DECL
   auto load_tile = [&](const CUtensorMap* tm, int row, int bh) -> bool {
     const uint32_t s = n_load % kStages;
@@ -262,31 +351,27 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     ++n_load;
     return true;
   };
+  auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
+  int item_loaded = -1;
   for (;;) {
-    const uint32_t r = n_rec % kRecords;
-    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 200, 0);                   // prof 0: no record yet
-    const Record& rec = sm.rec[r];
-    const int w = rec.work;
-    if (w < 0) break;
-    const int bh = w / p.Nq, i = w - bh * p.Nq;
-    const int j0 = rec.chunk * kBlk;
-    bool ok = true;
-    if (rec.flags & kRecFirst) {
-      SOL_WAIT(&sm.q_empty, (n_item & 1) ^ 1, 201, 2);                         // prof 2: Q slot busy
+    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                 // prof 0: no record yet
+    if (ev.type == kEvEnd) break;
+    if (ev.type == kEvAbort) { flag_abort(sm, p, 200); break; }
+    const int bh = ev.work / p.Nq, i = ev.work - bh * p.Nq;
+    if (ev.work != item_loaded) {
+      // Q_i for this work item (also for an item without tiles, to keep the phases in step)
+      if (!WAIT(&sm.q_empty, (n_item & 1) ^ 1, 2)) { flag_abort(sm, p, 201); break; }   // prof 2: Q slot busy
       mbar_arrive_expect_tx(&sm.q_full, kTileBytes);
       tma_load_3d(sQ, tm_q, &sm.q_full, 0, i * kBlk, bh);
       tma_load_3d(sQ + kHalfBytes, tm_q, &sm.q_full, 64, i * kBlk, bh);
       ++n_item;
+      item_loaded = ev.work;
     }
-    if (rec.flags & kRecApprox) ok = load_tile(tm_kc, j0, bh) && load_tile(tm_vm, j0, bh);
-    const int n_sel = rec.n_sel;
-    for (int e = 0; ok && e < n_sel; ++e) {
-      const int row = (j0 + rec.sel[e]) * kBlk;
-      ok = load_tile(tm_k, row, bh) && load_tile(tm_v, row, bh);
-    }
+    if (ev.type != kEvTile) continue;
+    bool ok;
+    if (ev.approx) ok = load_tile(tm_kc, ev.block, bh) && load_tile(tm_vm, ev.block, bh);
+    else ok = load_tile(tm_k, ev.block * kBlk, bh) && load_tile(tm_v, ev.block * kBlk, bh);
     if (!ok) { flag_abort(sm, p, 202); break; }
-    mbar_arrive(&sm.rec_empty[r]);
-    ++n_rec;
   }
   PROF_FLUSH(1);
   if (sm.abort_flag) {
@@ -300,137 +385,188 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
 }
 
 // ------------------------------------------------------------------------------------------------
-// mma issuer: one thread
-__device__ void mma_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV, uint32_t tmem) {
+// MMA issue is split over two single-thread roles so that neither the waits nor the scalar
+// bookkeeping of one kind of MMA delays the other; the tensor pipe arbitrates between them and all
+// ordering is carried by the mbarriers.
+//
+// Shared-memory descriptors: the upper word is constant (stride 1024 B between 8-row groups,
+// descriptor version, 128-byte swizzle); the lower word is (address >> 4) | (leading offset >> 4) << 16.
+__device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo) {
+  constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+
+// S_b = Q K^T (warp 10, one thread)
+__device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV, uint32_t tmem) {
   const uint32_t idesc_qk = make_idesc_bf16(kBlk, kBlk, false, false);
-  const uint32_t idesc_pv = make_idesc_bf16(kBlk, kD, false, true);
-  const uint32_t q_addr = smem_addr(sQ), kv_addr = smem_addr(sKV);
-  const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
-  uint32_t n_rec = 0, n_load = 0, n_item = 0, g = 0;   // g: tiles issued so far by this CTA
-  int tiles_in_item = 0;
+  const uint32_t q_lo = (smem_addr(sQ) >> 4) | (1u << 16);
+  const uint32_t kv_lo = (smem_addr(sKV) >> 4) | (1u << 16);
+  uint32_t n_item = 0, g = 0;
+  uint32_t slot = 0, slot_parity = 0;          // ring position of K(g): load 2g
+  Cursor cur;
   PROF_DECL
+  auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
+  bool ok = true;
+  int item_seen = -1;
   for (;;) {
-    const uint32_t r = n_rec % kRecords;
-    SOL_WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 300, 0);                   // prof 0: no record yet
-    const Record& rec = sm.rec[r];
-    if (rec.work < 0) break;
-    const uint8_t flags = rec.flags;
-    const int n_tiles = ((flags & kRecApprox) ? 1 : 0) + rec.n_sel;
-    mbar_arrive(&sm.rec_empty[r]);       // nothing else of the record is needed here
-    ++n_rec;
-    bool ok = true;
-    if (flags & kRecFirst) {
-      if (!WAIT(&sm.q_full, n_item & 1, 1)) { flag_abort(sm, p, 301); break; }      // prof 1: Q not loaded
+    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                       // prof 0: no record yet
+    if (ev.type == kEvAbort) { ok = false; break; }
+    if (ev.type == kEvEnd) break;
+    if (ev.work != item_seen) {
+      if (!WAIT(&sm.q_full, n_item & 1, 1)) { ok = false; break; }                    // prof 1: Q not loaded
       ++n_item;
-      tiles_in_item = 0;
+      item_seen = ev.work;
     }
-    for (int e = 0; e < n_tiles; ++e) {
-      // ---- S = Q K^T
-      const uint32_t sk = n_load % kStages;
-      if (!WAIT(&sm.kv_full[sk], (n_load / kStages) & 1, 2)) { ok = false; break; }   // prof 2: K not loaded
-      ++n_load;
-      if (g > 0 && !WAIT(&sm.pv_done, (g - 1) & 1, 3)) { ok = false; break; }         // prof 3: previous P V still running
-      tc_fence_after();
+    if (ev.type == kEvItemEnd) {                  // every MMA that reads Q_i has been issued
+      mma_commit(&sm.q_empty);
+      continue;
+    }
+    const uint32_t b = g & 1;
+    if (!WAIT(&sm.kv_full[slot], slot_parity, 2)) { ok = false; break; }              // prof 2: K not loaded
+    // the previous user of this score buffer was tile g-2: its P V must have read P out of it
+    if (g >= 2 && !WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }   // prof 3: score buffer busy
+    tc_fence_after();
+    {
+      PROF_T0
+      const uint32_t k_lo = kv_lo + slot * (kTileBytes >> 4);
+      const uint32_t d_tmem = tmem + kTmemS + b * kBlk;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
-        const uint32_t off = (ks / 4) * kHalfBytes + (ks % 4) * 32;
-        mma_ss(tmem_s, make_smem_desc_sw128(q_addr + off, 16, 1024),
-               make_smem_desc_sw128(kv_addr + sk * kTileBytes + off, 16, 1024), idesc_qk, ks > 0);
+        const uint32_t off = ((ks / 4) * kHalfBytes + (ks % 4) * 32) >> 4;
+        mma_ss(d_tmem, desc_from_lo(q_lo + off), desc_from_lo(k_lo + off), idesc_qk, ks > 0);
       }
-      mma_commit(&sm.kv_empty[sk]);
-      mma_commit(&sm.s_full);
-      // ---- O += P V
-      const uint32_t sv = n_load % kStages;
-      if (!WAIT(&sm.kv_full[sv], (n_load / kStages) & 1, 4)) { ok = false; break; }   // prof 4: V not loaded
-      ++n_load;
-      if (!WAIT(&sm.p_full, g & 1, 5)) { ok = false; break; }                         // prof 5: softmax not done
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < kBlk / 16; ++ks) {
-        mma_ts(tmem_o, tmem_s + ks * 8, make_smem_desc_sw128(kv_addr + sv * kTileBytes + ks * 2048, kHalfBytes, 1024),
-               idesc_pv, (tiles_in_item > 0 || ks > 0) ? 1u : 0u);
-      }
-      mma_commit(&sm.kv_empty[sv]);
-      mma_commit(&sm.pv_done);
-      ++g;
-      ++tiles_in_item;
+      mma_commit(&sm.kv_empty[slot]);
+      mma_commit(&sm.s_full[b]);
+      PROF_ADD(6)                                                                      // prof 6: issuing Q K^T
     }
-    if (!ok) { flag_abort(sm, p, 302); break; }
-    if (flags & kRecLast) mma_commit(&sm.q_empty);     // every MMA that reads Q_i has been issued
+    ++g;
+    slot += 2;                                    // K tiles sit at every other ring position
+    if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
   }
+  if (!ok) flag_abort(sm, p, 300);
   PROF_FLUSH(2);
 }
 
+// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11, one thread)
+__device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uint32_t tmem) {
+  const uint32_t idesc_pv = make_idesc_bf16(kBlk, kD, false, true);
+  const uint32_t kv_lo = (smem_addr(sKV) >> 4) | ((uint32_t)(kHalfBytes >> 4) << 16);
+  uint32_t g = 0;
+  uint32_t slot = 1, slot_parity = 0;          // ring position of V(g): load 2g+1
+  Cursor cur;
+  auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
+  bool ok = true;
+  for (;;) {
+    const Event ev = next_event(sm, cur, nullptr, release);
+    if (ev.type == kEvAbort) { ok = false; break; }
+    if (ev.type == kEvEnd) break;
+    if (ev.type != kEvTile) continue;
+    const uint32_t b = g & 1;
+    if (!mbar_wait(&sm.kv_full[slot], slot_parity, &sm.abort_flag)) { ok = false; break; }
+    const uint32_t v_lo = kv_lo + slot * (kTileBytes >> 4);
+    const uint32_t acc_first = ev.first ? 0u : 1u;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < kHalf / 16; ++ks) {
+        mma_ts(tmem + kTmemO + h * kD, tmem + kTmemS + b * kBlk + h * kHalf + ks * 8,
+               desc_from_lo(v_lo + ((h * (kHalf * 128) + ks * 2048) >> 4)), idesc_pv, ks > 0 ? 1u : acc_first);
+      }
+    }
+    if (!ok) break;
+    mma_commit(&sm.kv_empty[slot]);
+    mma_commit(&sm.pv_done[b]);
+    ++g;
+    slot += 2;
+    if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
+  }
+  if (!ok) flag_abort(sm, p, 301);
+}
+
 // ------------------------------------------------------------------------------------------------
-// softmax + correction + epilogue: 128 threads, thread = query row
-__device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int warp, int lane) {
+// softmax + correction + epilogue: two warpgroups of 128 threads; thread = query row, warpgroup h
+// owns key columns [64h, 64h+64) of every tile
+__device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, int warp_in_group, int lane) {
   const unsigned full = 0xffffffffu;
-  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-  const uint32_t t_s = lane_base, t_o = lane_base + 128;
-  const int row = warp * 32 + lane;
+  const uint32_t lane_base = tmem + ((uint32_t)(warp_in_group * 32) << 16);
+  const uint32_t t_o = lane_base + kTmemO + h * kD;          // this group's accumulator
+  const uint32_t t_o_other = lane_base + kTmemO + (1 - h) * kD;
+  const int row = warp_in_group * 32 + lane;
   const float sl2 = p.scale * 1.4426950408889634f;
   const float inv_sl2 = 1.f / sl2;
-  uint32_t n_rec = 0, g = 0;
-  int tiles_in_item = 0;
-  float m_used = 0.f, l = 0.f;
-  bool alive = true;
+  uint32_t g = 0, n_merge = 0;
+  bool stagger = true;
+  float m_used = -INFINITY, l = 0.f;
+  Cursor cur;
   PROF_DECL
-  while (alive) {
-    const uint32_t r = n_rec % kRecords;
-    if (!WAIT(&sm.rec_full[r], (n_rec / kRecords) & 1, 0)) { flag_abort(sm, p, 400); break; }   // prof 0: no record yet
-    const Record& rec = sm.rec[r];
-    const int w = rec.work;
-    if (w < 0) break;
-    const uint8_t flags = rec.flags;
-    const int n_sel = rec.n_sel;
-    const int n_tiles = ((flags & kRecApprox) ? 1 : 0) + n_sel;
-    const int j0 = rec.chunk * kBlk;
-    if (flags & kRecFirst) tiles_in_item = 0;
-    for (int e = 0; e < n_tiles; ++e) {
-      const bool approx = (flags & kRecApprox) && e == 0;
-      int cols_valid = kBlk;
-      if (!approx) {
-        const int j = j0 + rec.sel[e - ((flags & kRecApprox) ? 1 : 0)];
-        cols_valid = min(kBlk, p.N - j * kBlk);
+  auto release = [&](uint32_t r) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.rec_empty[r]);
+  };
+  for (;;) {
+    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                       // prof 0: no record yet
+    if (ev.type == kEvEnd) break;
+    if (ev.type == kEvAbort) { flag_abort(sm, p, 400); break; }
+
+    if (ev.type == kEvTile) {
+      if (stagger) {
+        // The two groups leave the end-of-item rendezvous in lockstep and would then hit the MUFU
+        // unit in the same phase of every tile; holding group 1 back by about half a tile keeps
+        // one group's exponentials under the other's loads, maxima and stores.
+        stagger = false;
+        if (h == 1 && kStaggerCycles > 0) {
+          const long long t_start = clock64();
+          while (clock64() - t_start < kStaggerCycles) {}
+        }
       }
+      const uint32_t b = g & 1;
+      const uint32_t t_s = lane_base + kTmemS + b * kBlk + h * kHalf;
+      const bool approx = ev.approx;
+      const int cols_valid = approx ? kBlk : min(kBlk, p.N - ev.block * kBlk);
       const bool general = approx || cols_valid < kBlk;
-      if (!WAIT(&sm.s_full, g & 1, 1)) { flag_abort(sm, p, 401); alive = false; break; }   // prof 1: S not ready
+      if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
       tc_fence_after();
-      // ---- the whole row of S (128 fp32) into registers with one wait
-      uint32_t sr[kBlk];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+      // ---- this group's half row of S (64 fp32) into registers with one wait
+      uint32_t sr[kHalf];
+      PROF_T0
+      tmem_ld_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+      tmem_ld_32x32b_x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       tmem_ld_wait();
+      PROF_ADD(7)                                                                      // prof 7: loading S
       if (general) {
         // bring the rare tiles (approximate chunk, ragged last block) to the common form
         // logit = sl2 * x by folding the column bias into x; -inf marks masked columns
 #pragma unroll
-        for (int c = 0; c < kBlk; ++c) {
+        for (int c = 0; c < kHalf; ++c) {
           const float x = __uint_as_float(sr[c]);
-          sr[c] = __float_as_uint(approx ? fmaf(rec.bias[c], inv_sl2, x) : (c < cols_valid ? x : -INFINITY));
+          const int col = h * kHalf + c;
+          sr[c] = __float_as_uint(approx ? fmaf(ev.rec->bias[col], inv_sl2, x) : (col < cols_valid ? x : -INFINITY));
         }
       }
       float mx;
       {
         float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
+        for (int c = 0; c < 16; ++c) {
           m0 = fmaxf(m0, __uint_as_float(sr[c]));
-          m1 = fmaxf(m1, __uint_as_float(sr[32 + c]));
-          m2 = fmaxf(m2, __uint_as_float(sr[64 + c]));
-          m3 = fmaxf(m3, __uint_as_float(sr[96 + c]));
+          m1 = fmaxf(m1, __uint_as_float(sr[16 + c]));
+          m2 = fmaxf(m2, __uint_as_float(sr[32 + c]));
+          m3 = fmaxf(m3, __uint_as_float(sr[48 + c]));
         }
-        mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sl2;
+        mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sl2;       // -inf when the whole half is masked
       }
-      // ---- running maximum, lazy rescale of O
-      if (tiles_in_item == 0) {
+      // ---- running maximum, lazy rescale of O_h
+      if (ev.first) {
         m_used = mx;
         l = 0.f;
       } else if (__any_sync(full, mx > m_used + kRescaleThreshold)) {
         const float m_new = fmaxf(m_used, mx);
-        const float f = ex2(m_used - m_new);
-        PROF_COUNT(4);                                                                   // prof 4: number of rescales
-        if (!WAIT(&sm.pv_done, (g - 1) & 1, 2)) { flag_abort(sm, p, 402); alive = false; break; }
+        const float f = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
+        PROF_COUNT(4);                                                                  // prof 4: number of rescales
+        // P V of the previous tile must have landed in O_h
+        if (!WAIT(&sm.pv_done[b ^ 1], ((g - 1) >> 1) & 1, 2)) { flag_abort(sm, p, 402); break; }
         tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -445,12 +581,12 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
         m_used = m_new;
       }
       // ---- P = exp2(sl2 * S - m): most elements on the MUFU unit, every kPolyEvery-th one as a
-      //      polynomial on the FMA pipe; row sum; P (bf16) back to TMEM over the first half of S
+      //      polynomial on the FMA pipe; row sum; P (bf16) back to TMEM over the start of the half
       {
-        const float nm = -m_used;
+        const float nm = (m_used == -INFINITY) ? 0.f : -m_used;   // a half that has seen nothing yet: all P = 0
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < kBlk; c += 4) {
+        for (int c = 0; c < kHalf; c += 4) {
           float e[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -465,60 +601,79 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int war
         }
         l += (sum0 + sum1) + (sum2 + sum3);
         tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-        tmem_st_32x32b_x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       }
+      PROF_ADD(8)                                                                      // prof 8: load + arithmetic
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(&sm.p_full);
-      PROF_COUNT(5);                                                                     // prof 5: tiles
+      mbar_arrive(&sm.p_full[h][b]);
+      PROF_ADD(9)                                                                      // prof 9: whole tile
+      PROF_COUNT(5);                                                                    // prof 5: tiles
       ++g;
-      ++tiles_in_item;
+      continue;
     }
-    if (!alive) break;
-    // ---- end of the work item: O_i = acc / l
-    if (flags & kRecLast) {
-      const int bh = w / p.Nq, i = w - bh * p.Nq;
-      const int q_rows = min(kBlk, p.N - i * kBlk);
-      __nv_bfloat16* orow = p.out + ((size_t)bh * p.N + (size_t)i * kBlk + row) * kD;
-      if (tiles_in_item > 0) {
-        if (!WAIT(&sm.pv_done, (g - 1) & 1, 3)) { flag_abort(sm, p, 403); break; }           // prof 3: last P V of the item
-        tc_fence_after();
-        const float inv = 1.f / l;
+
+    // ---- end of the work item: merge the two partial results, O_i = (w0 O0 + w1 O1) / (w0 l0 + w1 l1)
+    const int bh = ev.work / p.Nq, i = ev.work - bh * p.Nq;
+    const int q_rows = min(kBlk, p.N - i * kBlk);
+    __nv_bfloat16* orow = p.out + ((size_t)bh * p.N + (size_t)i * kBlk + row) * kD + h * kHalf;
+    if (!ev.first) {
+      // the last P V of the item (one commit covers both halves)
+      if (!WAIT(&sm.pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, 3)) { flag_abort(sm, p, 403); break; }   // prof 3
+      tc_fence_after();
+      sm.ml[h][row] = make_float2(m_used, l);
+      mbar_arrive(&sm.x_full);
+      if (!WAIT(&sm.x_full, n_merge & 1, 6)) { flag_abort(sm, p, 404); break; }       // prof 6: other group not done
+      const float2 other = sm.ml[1 - h][row];
+      const float m = fmaxf(m_used, other.x);
+      const float w_own = (m_used == -INFINITY) ? 0.f : ex2(m_used - m);
+      const float w_other = (other.x == -INFINITY) ? 0.f : ex2(other.x - m);
+      const float inv = 1.f / (l * w_own + other.y * w_other);
+      const float c_own = w_own * inv, c_other = w_other * inv;
+      // this thread writes channels [64h, 64h+64) of its row
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t o[32];
-          tmem_ld_32x32b_x32(t_o + c * 32, o);
-          tmem_ld_wait();
-          if (row < q_rows) {
+      for (int c = 0; c < 2; ++c) {
+        uint32_t a[32], bb[32];
+        tmem_ld_32x32b_x32(t_o + h * kHalf + c * 32, a);
+        tmem_ld_32x32b_x32(t_o_other + h * kHalf + c * 32, bb);
+        tmem_ld_wait();
+        if (row < q_rows) {
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              uint4 pk;
-              uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
+          for (int x = 0; x < 4; ++x) {
+            uint4 pk;
+            uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
 #pragma unroll
-              for (int y = 0; y < 4; ++y) {
-                __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[x * 8 + 2 * y]) * inv,
-                                                          __uint_as_float(o[x * 8 + 2 * y + 1]) * inv);
-                pw[y] = *reinterpret_cast<uint32_t*>(&hh);
-              }
-              *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = pk;
+            for (int y = 0; y < 4; ++y) {
+              const int e0 = x * 8 + 2 * y;
+              // a partial accumulator that never received a tile may hold anything: weight 0 must win
+              const float v0 = (w_own > 0.f ? __uint_as_float(a[e0]) * c_own : 0.f) +
+                               (w_other > 0.f ? __uint_as_float(bb[e0]) * c_other : 0.f);
+              const float v1 = (w_own > 0.f ? __uint_as_float(a[e0 + 1]) * c_own : 0.f) +
+                               (w_other > 0.f ? __uint_as_float(bb[e0 + 1]) * c_other : 0.f);
+              __nv_bfloat162 hh = __floats2bfloat162_rn(v0, v1);
+              pw[y] = *reinterpret_cast<uint32_t*>(&hh);
             }
+            *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = pk;
           }
         }
-        tc_fence_before();
-      } else if (row < q_rows) {
-        // a query block that routed nothing in keep-or-drop mode has no attention mass at all
-        for (int c = 0; c < kD; c += 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
       }
-      tiles_in_item = 0;
+      tc_fence_before();
+      // neither group may start the next item (whose first P V overwrites O0 / O1) before both
+      // have finished reading
+      mbar_arrive(&sm.x_done);
+      if (!WAIT(&sm.x_done, n_merge & 1, 6)) { flag_abort(sm, p, 405); break; }
+      ++n_merge;
+      stagger = true;
+    } else if (row < q_rows) {
+      // a query block that routed nothing in keep-or-drop mode has no attention mass at all
+      for (int c = 0; c < kHalf; c += 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.rec_empty[r]);
-    ++n_rec;
+    m_used = -INFINITY;
+    l = 0.f;
   }
-  if (lane == 0 && warp == 0) PROF_FLUSH(3);
+  if (lane == 0 && warp_in_group == 0 && h == 0) PROF_FLUSH(3);
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kc,
                  const __grid_constant__ CUtensorMap tm_vm, const Params p) {
@@ -531,13 +686,20 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     sm.abort_flag = 0;
-    for (int r = 0; r < kRecords; ++r) { mbar_init(&sm.rec_full[r], 1); mbar_init(&sm.rec_empty[r], 6); }
+    // a record is released by the producer, the two MMA threads and the 8 softmax warps
+    for (int r = 0; r < kRecords; ++r) { mbar_init(&sm.rec_full[r], 1); mbar_init(&sm.rec_empty[r], 11); }
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
     mbar_init(&sm.q_full, 1); mbar_init(&sm.q_empty, 1);
-    mbar_init(&sm.s_full, 1); mbar_init(&sm.p_full, 128); mbar_init(&sm.pv_done, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm.s_full[b], 1);
+      mbar_init(&sm.pv_done[b], 1);
+      mbar_init(&sm.p_full[0][b], 128);
+      mbar_init(&sm.p_full[1][b], 128);
+    }
+    mbar_init(&sm.x_full, 256); mbar_init(&sm.x_done, 256);
     fence_mbar_init();
   }
-  if (warp == 5 && lane == 0) {
+  if (warp == 9 && lane == 0) {
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
     prefetch_tensormap(&tm_kc); prefetch_tensormap(&tm_vm);
   }
@@ -547,18 +709,16 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp < 4) {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-    softmax_role(sm, p, tmem, warp, lane);
-  } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
-  }
-  if (warp == 4) {
+  if (warp < 8) {
+    softmax_role(sm, p, tmem, warp / 4, warp % 4, lane);
+  } else if (warp == 8) {
     router_role(sm, p, lane);
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     if (lane == 0) producer_role(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
-  } else if (warp == 6) {
-    if (lane == 0) mma_role(sm, p, sQ, sKV, tmem);
+  } else if (warp == 10) {
+    if (lane == 0) mma_qk_role(sm, p, sQ, sKV, tmem);
+  } else {
+    if (lane == 0) mma_pv_role(sm, p, sKV, tmem);
   }
   tc_fence_before();
   __syncthreads();
@@ -601,7 +761,7 @@ cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __n
   const size_t smem = 1024 + kTileBytes + kStages * kTileBytes + sizeof(Shared);
   e = cudaFuncSetAttribute(fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int grid = prm.total_work < 2 * sms ? prm.total_work : 2 * sms;
+  const int grid = prm.total_work < sms ? prm.total_work : sms;
   fwd_sm100_kernel<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
   if (n_launches) *n_launches += 1;
   return cudaGetLastError();
