@@ -15,6 +15,7 @@ constexpr int kStatusWords = 16;      // int32 words at the start of the workspa
 constexpr int kStatusDevice = 0;      // word 0: device status (0 ok, SOL_ERR_DEVICE_TIMEOUT ...)
 constexpr int kStatusDetail = 1;      // word 1: where a bounded wait gave up (debug aid)
 constexpr int kStatusTileCounter = 2; // word 2: persistent-kernel work counter
+constexpr int kCovSlices = 4;         // partial second-moment matrices per (batch, head)
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -37,7 +38,7 @@ struct WsLayout {
   size_t kcb;     // bf16 [BH][Nk][d]   KC rounded, MMA operand of the approximate branch
   size_t vmb;     // bf16 [BH][Nk][d]   VC / n_j rounded, MMA operand of the approximate branch
   size_t mk;      // fp32 [BH][d]       first moment of the pooled keys (Eq. 5)
-  size_t covk;    // fp32 [BH][d][d]    centred second moment of the pooled keys (Eq. 5)
+  size_t covk;    // fp32 [kCovSlices][BH][d][d]  partial centred second moments of the pooled keys (Eq. 5)
   size_t mu, sigma, tau;  // fp32 [BH][Nq] each (Eq. 4)
   size_t total;
 };
@@ -53,7 +54,7 @@ inline WsLayout make_layout(int BH, int Nq, int Nk, int d) {
   w.kcb = take(2 * (size_t)BH * Nk * d);
   w.vmb = take(2 * (size_t)BH * Nk * d);
   w.mk = take(sizeof(float) * (size_t)BH * d);
-  w.covk = take(sizeof(float) * (size_t)BH * d * d);
+  w.covk = take(sizeof(float) * (size_t)kCovSlices * BH * d * d);
   w.mu = take(sizeof(float) * (size_t)BH * Nq);
   w.sigma = take(sizeof(float) * (size_t)BH * Nq);
   w.tau = take(sizeof(float) * (size_t)BH * Nq);

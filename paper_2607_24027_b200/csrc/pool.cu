@@ -99,29 +99,33 @@ pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
   }
 }
 
-// First moment of the pooled keys, m_K = (1/Nk) sum_j KC_j  (Eq. 5).  One CTA per (batch, head),
-// thread c owns channel c.
+// First moment of the pooled keys, m_K = (1/Nk) sum_j KC_j  (Eq. 5).  One CTA per (batch, head):
+// 4 row groups x D channels, combined through shared memory.
 template <int D>
-__global__ void __launch_bounds__(D) key_mean_kernel(WsPtrs ws, int Nk) {
-  const int bh = blockIdx.x, c = threadIdx.x;
+__global__ void __launch_bounds__(4 * D) key_mean_kernel(WsPtrs ws, int Nk) {
+  __shared__ float part[4][D];
+  const int bh = blockIdx.x, c = threadIdx.x % D, grp = threadIdx.x / D;
   const float* kc = ws.kc + (size_t)bh * Nk * D;
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-  int j = 0;
-  for (; j + 3 < Nk; j += 4) {
+  float s0 = 0.f, s1 = 0.f;
+  int j = grp;
+  for (; j + 4 < Nk; j += 8) {
     s0 += kc[(size_t)j * D + c];
-    s1 += kc[(size_t)(j + 1) * D + c];
-    s2 += kc[(size_t)(j + 2) * D + c];
-    s3 += kc[(size_t)(j + 3) * D + c];
+    s1 += kc[(size_t)(j + 4) * D + c];
   }
-  for (; j < Nk; ++j) s0 += kc[(size_t)j * D + c];
-  ws.mk[(size_t)bh * D + c] = ((s0 + s1) + (s2 + s3)) / (float)Nk;
+  if (j < Nk) s0 += kc[(size_t)j * D + c];
+  part[grp][c] = s0 + s1;
+  __syncthreads();
+  if (grp == 0) ws.mk[(size_t)bh * D + c] = ((part[0][c] + part[1][c]) + (part[2][c] + part[3][c])) / (float)Nk;
 }
 
 // Centred second moment of the pooled keys,
 //   C_K = (1/Nk) sum_j (KC_j - m_K)^T (KC_j - m_K)  =  (1/Nk) sum_j KC_j^T KC_j - m_K^T m_K,
 // i.e. the bracket of Eq. (5) with the mu_i^2 term already folded in, which avoids the
-// cancellation of the uncentred form in fp32.  Grid (D/16, BH); a CTA of 256 threads owns 16
-// rows of C_K, thread (r, cg) owns C_K[r][cg*8 .. cg*8+7].
+// cancellation of the uncentred form in fp32.  Grid (D/16, BH, key slices); a CTA of 256 threads
+// owns 16 rows of C_K for one slice of the pooled keys, thread (r, cg) owns C_K[r][cg*8 ..
+// cg*8+7]; every slice writes its own partial matrix (covk holds kCovSlices of them per launch,
+// slice-major) and tau_kernel adds them in a fixed order, so the result is bit-stable run to run.
+
 template <int D>
 __global__ void __launch_bounds__(256) key_cov_kernel(WsPtrs ws, int Nk) {
   constexpr int ROWS = 16;
@@ -134,11 +138,13 @@ __global__ void __launch_bounds__(256) key_cov_kernel(WsPtrs ws, int Nk) {
   const int c0 = (threadIdx.x % CG) * CPT;
   const float* kc = ws.kc + (size_t)bh * Nk * D;
   const float* mk = ws.mk + (size_t)bh * D;
+  const int per_slice = ceil_div(Nk, kCovSlices);
+  const int j_begin = blockIdx.z * per_slice, j_end = min(Nk, j_begin + per_slice);
   float acc[CPT];
 #pragma unroll
   for (int c = 0; c < CPT; ++c) acc[c] = 0.f;
-  for (int j0 = 0; j0 < Nk; j0 += JT) {
-    const int nj = min(JT, Nk - j0);
+  for (int j0 = j_begin; j0 < j_end; j0 += JT) {
+    const int nj = min(JT, j_end - j0);
     for (int e = threadIdx.x; e < nj * D; e += 256) {
       const int jj = e / D, c = e % D;
       xs[jj][c] = kc[(size_t)(j0 + jj) * D + c] - mk[c];
@@ -151,46 +157,76 @@ __global__ void __launch_bounds__(256) key_cov_kernel(WsPtrs ws, int Nk) {
     }
     __syncthreads();
   }
-  float* cov = ws.covk + ((size_t)bh * D + r) * D + c0;
+  float* cov = ws.covk + (((size_t)blockIdx.z * gridDim.y + bh) * D + r) * D + c0;
 #pragma unroll
   for (int c = 0; c < CPT; ++c) cov[c] = acc[c] / (float)Nk;
 }
 
 // Per-query-block statistics and threshold (Eq. 4, Eq. 5):
 //   mu_i = s * Qbar_i . m_K,   sigma_i^2 = s^2 * Qbar_i C_K Qbar_i^T,   tau_i = mu_i + beta sigma_i.
-// Grid (ceil(Nq / 64), BH); C_K is staged in shared memory once per CTA; each of the 8 warps
-// handles 8 query blocks.
+// Grid (ceil(Nq / 64), BH).  A CTA stages C_K and 64 pooled queries in shared memory and forms
+// Y = Qbar C_K as a register-tiled product (thread (rg, cg): 4 query blocks x 8 channels); the
+// quadratic form is the row sum of Y o Qbar, reduced over the 16 threads of a query-block group.
 template <int D>
 __global__ void __launch_bounds__(256) tau_kernel(WsPtrs ws, int Nq, float scale, float beta) {
-  extern __shared__ float cov_s[];               // [D][D+1]
-  constexpr int LD = D + 1;
-  constexpr int PER = D / 32;                    // channels per lane
-  const int bh = blockIdx.y;
+  extern __shared__ float smem_f[];
+  constexpr int QT = 64;                         // query blocks per CTA
+  constexpr int CPT = D / 16;                    // channels per thread (8 or 4)
+  float* cov_s = smem_f;                         // [D][D]
+  float* q_s = smem_f + D * D;                   // [QT][D + 1]
+  constexpr int QLD = D + 1;
+  const int bh = blockIdx.y, i0 = blockIdx.x * QT;
+  const size_t slice_stride = (size_t)gridDim.y * D * D;
   const float* cov = ws.covk + (size_t)bh * D * D;
-  for (int e = threadIdx.x; e < D * D; e += 256) cov_s[(e / D) * LD + (e % D)] = cov[e];
+  for (int e = threadIdx.x; e < D * D / 4; e += 256) {
+    float4 a = reinterpret_cast<const float4*>(cov)[e];
+#pragma unroll
+    for (int sl = 1; sl < kCovSlices; ++sl) {
+      const float4 b = reinterpret_cast<const float4*>(cov + sl * slice_stride)[e];
+      a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    reinterpret_cast<float4*>(cov_s)[e] = a;
+  }
+  for (int e = threadIdx.x; e < QT * D; e += 256) {
+    const int rq = e / D, c = e % D;
+    q_s[rq * QLD + c] = (i0 + rq < Nq) ? ws.qbar[((size_t)bh * Nq + i0 + rq) * D + c] : 0.f;
+  }
   __syncthreads();
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int rg = threadIdx.x / 16, cg = threadIdx.x % 16;
+  const int c0 = cg * CPT;
+  float y[4][CPT];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) y[a][c] = 0.f;
+  for (int k = 0; k < D; ++k) {
+    float qa[4], cb[CPT];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) qa[a] = q_s[(rg * 4 + a) * QLD + k];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) cb[c] = cov_s[k * D + c0 + c];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int c = 0; c < CPT; ++c) y[a][c] = fmaf(qa[a], cb[c], y[a][c]);
+  }
   const float* mk = ws.mk + (size_t)bh * D;
-  for (int t = 0; t < 8; ++t) {
-    const int i = blockIdx.x * 64 + warp * 8 + t;
-    if (i >= Nq) break;
-    const float* qb = ws.qbar + ((size_t)bh * Nq + i) * D;
-    // lane owns rows lane, lane+32, ... of C_K; y_r = sum_c C[r][c] q[c]; quad = sum_r q[r] y_r
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
     float quad = 0.f, dotm = 0.f;
 #pragma unroll
-    for (int rr = 0; rr < PER; ++rr) {
-      const int r = lane + 32 * rr;
-      float y = 0.f;
-      for (int c = 0; c < D; ++c) y = fmaf(cov_s[r * LD + c], qb[c], y);
-      quad = fmaf(qb[r], y, quad);
-      dotm = fmaf(qb[r], mk[r], dotm);
+    for (int c = 0; c < CPT; ++c) {
+      const float qv = q_s[(rg * 4 + a) * QLD + c0 + c];
+      quad = fmaf(y[a][c], qv, quad);
+      dotm = fmaf(qv, mk[c0 + c], dotm);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = 8; o > 0; o >>= 1) {
       quad += __shfl_xor_sync(0xffffffffu, quad, o);
       dotm += __shfl_xor_sync(0xffffffffu, dotm, o);
     }
-    if (lane == 0) {
+    const int i = i0 + rg * 4 + a;
+    if (cg == 0 && i < Nq) {
       const float mu = scale * dotm;
       const float sigma = scale * sqrtf(fmaxf(quad, 0.f));
       float tau;
@@ -223,15 +259,11 @@ cudaError_t launch_pool(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
 
 template <int D>
 static cudaError_t thresholds_impl(const Problem& p, const WsPtrs& ws, cudaStream_t stream, int* n_launches) {
-  key_mean_kernel<D><<<p.BH, D, 0, stream>>>(ws, p.Nk);
-  key_cov_kernel<D><<<dim3(D / 16, p.BH), 256, 0, stream>>>(ws, p.Nk);
-  const size_t smem = sizeof(float) * D * (D + 1);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tau_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  key_mean_kernel<D><<<p.BH, 4 * D, 0, stream>>>(ws, p.Nk);
+  key_cov_kernel<D><<<dim3(D / 16, p.BH, kCovSlices), 256, 0, stream>>>(ws, p.Nk);
+  const size_t smem = sizeof(float) * (D * D + 64 * (D + 1));
+  cudaError_t e = cudaFuncSetAttribute(tau_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
   tau_kernel<D><<<dim3(ceil_div(p.Nq, 64), p.BH), 256, smem, stream>>>(ws, p.Nq, p.scale, p.beta);
   if (n_launches) *n_launches += 3;
   return cudaGetLastError();
