@@ -47,7 +47,8 @@ enum {
   SOL_ERR_UNSUPPORTED_ARCH  = -3,  /* current device is not compute capability 10.x            */
   SOL_ERR_WORKSPACE         = -4,  /* no workspace bound / workspace too small or misaligned   */
   SOL_ERR_CUDA              = -5,  /* a CUDA runtime or driver call failed (launch, tensor map)*/
-  SOL_ERR_DEVICE_TIMEOUT    = -6   /* a bounded device-side wait expired; output is invalid    */
+  SOL_ERR_DEVICE_TIMEOUT    = -6,  /* a bounded device-side wait expired; output is invalid    */
+  SOL_ERR_SCRATCH_LIMIT     = -7   /* problem larger than the library's built-in scratch array */
 };
 
 /* what the fused kernel computes */
@@ -74,7 +75,7 @@ const char* sol_attn_status_string(sol_status_t status);
 size_t sol_attn_workspace_bytes(int B, int H, int N, int d, int block_q, int block_k);
 
 /* Byte offsets of the parity-relevant arrays inside a workspace laid out for the given problem.
- * All arrays are fp32 except counts_unused.  qbar: [B,H,Nq,d] mean of each query block;
+ * All arrays are fp32.  qbar: [B,H,Nq,d] mean of each query block;
  * kc: [B,H,Nk,d] mean of each key block; vc: [B,H,Nk,d] SUM of each value block;
  * mu, sigma, tau: [B,H,Nq]; status: int32[16] (word 0 = device status, see below). */
 typedef struct {
@@ -146,6 +147,34 @@ sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* h
 /* Synchronises `stream`, then returns the device status word of the bound workspace
  * (SOL_OK, or SOL_ERR_DEVICE_TIMEOUT when a kernel gave up on a bounded wait) and clears it. */
 sol_status_t sol_attn_read_device_status(sol_stream_t stream);
+
+/* Threshold step for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is an interface variant, it computes the same mu, sigma, tau of Eq. 4 / Eq. 5.)
+ *
+ * Who needs it: code that is handed only its inputs and outputs -- an operator running inside
+ * another framework's memory pool, a process whose device memory was reserved up front, a
+ * serving loop in which an allocation would synchronise the device.  Such callers cannot provide
+ * the workspace the other entry points keep the pooled-key moments in, so here the moments live
+ * in a fixed array inside the library image: 4 MiB of device memory on every GPU that loads the
+ * library, from load until exit.
+ *
+ *   qbar   device fp32 [B,H,Nq,d]  mean of each query block (as produced by sol_attn_pool)
+ *   kc     device fp32 [B,H,Nk,d]  mean of each key block
+ *   mu, sigma, tau   device fp32 [B,H,Nq] outputs, owned by the caller
+ *   scale  logit scale, <= 0 selects 1/sqrt(d);  threshold = beta
+ *
+ * Limit: B*H*d*(d+1) <= sol_attn_thresholds_static_max_floats() (2^20), i.e. B*H <= 63 for d = 128
+ * and B*H <= 252 for d = 64; larger problems return SOL_ERR_SCRATCH_LIMIT and launch nothing.
+ * The call allocates and frees nothing, enqueues three kernels on `stream` and returns.
+ * The first call on each device looks up the array's device address (a runtime query, not an
+ * allocation); make that first call outside any stream capture.
+ * All calls on a device share the one array and every call overwrites the part it uses before
+ * reading it, so nothing needs clearing between calls -- but two calls that overlap on the GPU
+ * (different streams, no ordering) race on it and must be serialised by the caller. */
+sol_status_t sol_attn_thresholds_static(const float* qbar, const float* kc, int B, int H, int Nq, int Nk,
+                                        int d, float scale, float threshold,
+                                        float* mu, float* sigma, float* tau, sol_stream_t stream);
+size_t sol_attn_thresholds_static_max_floats(void);
 
 /* Number of kernels the library has launched since it was loaded (for launch accounting). */
 int64_t sol_attn_launch_count(void);

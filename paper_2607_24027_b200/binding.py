@@ -23,6 +23,7 @@ SOL_ERR_UNSUPPORTED_ARCH = -3
 SOL_ERR_WORKSPACE = -4
 SOL_ERR_CUDA = -5
 SOL_ERR_DEVICE_TIMEOUT = -6
+SOL_ERR_SCRATCH_LIMIT = -7
 
 SOL_MODE_SOL, SOL_MODE_DENSE, SOL_MODE_EXACT_ONLY = 0, 1, 2
 SOL_IMPL_AUTO, SOL_IMPL_TCGEN05, SOL_IMPL_MMA_SYNC = 0, 1, 2
@@ -31,7 +32,7 @@ EXPORTS = [
     "sol_attn_status_string", "sol_attn_workspace_bytes", "sol_attn_workspace_view",
     "sol_attn_bind_workspace", "sol_attn_pool", "sol_attn_forward", "sol_attn_dense",
     "sol_attn_forward_ex", "sol_attn_forward_host", "sol_attn_read_device_status",
-    "sol_attn_launch_count",
+    "sol_attn_launch_count", "sol_attn_thresholds_static", "sol_attn_thresholds_static_max_floats",
 ]
 
 
@@ -95,6 +96,11 @@ def lib() -> ctypes.CDLL:
     L.sol_attn_read_device_status.argtypes = [ctypes.c_void_p]
     L.sol_attn_launch_count.restype = ctypes.c_int64
     L.sol_attn_launch_count.argtypes = []
+    L.sol_attn_thresholds_static.restype = ctypes.c_int32
+    L.sol_attn_thresholds_static.argtypes = [ctypes.c_void_p] * 2 + [ctypes.c_int] * 5 + [ctypes.c_float] * 2 + \
+                                            [ctypes.c_void_p] * 4
+    L.sol_attn_thresholds_static_max_floats.restype = ctypes.c_size_t
+    L.sol_attn_thresholds_static_max_floats.argtypes = []
     _lib = L
     return L
 
@@ -231,6 +237,23 @@ def sol_attn_forward_host(hq, hk, hv, hout, dq, dk, dv, dout, block_q, block_k, 
                                        _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dout), B, H, N, d,
                                        block_q, block_k, float(threshold), _stream(stream)),
            "sol_attn_forward_host")
+
+
+def sol_attn_thresholds_static(qbar, kc, threshold, mu, sigma, tau, scale=0.0, stream=None):
+    """mu, sigma, tau (fp32 [B, H, Nq], caller-owned) from pooled queries / keys (fp32 [B, H, N*, d]) without
+    any device allocation: the pooled-key moments go to an array built into the library."""
+    B, H, Nq, d = (int(x) for x in qbar.shape)
+    Nk = int(kc.shape[2])
+    for t in (qbar, kc, mu, sigma, tau):
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("expected contiguous CUDA fp32 tensors")
+    _check(lib().sol_attn_thresholds_static(_ptr(qbar), _ptr(kc), B, H, Nq, Nk, d, float(scale), float(threshold),
+                                            _ptr(mu), _ptr(sigma), _ptr(tau), _stream(stream)),
+           "sol_attn_thresholds_static")
+
+
+def sol_attn_thresholds_static_max_floats() -> int:
+    return int(lib().sol_attn_thresholds_static_max_floats())
 
 
 def sol_attn_read_device_status(stream=None) -> int:

@@ -73,6 +73,7 @@ const char* sol_attn_status_string(sol_status_t s) {
     case SOL_ERR_WORKSPACE: return "SOL_ERR_WORKSPACE";
     case SOL_ERR_CUDA: return "SOL_ERR_CUDA";
     case SOL_ERR_DEVICE_TIMEOUT: return "SOL_ERR_DEVICE_TIMEOUT";
+    case SOL_ERR_SCRATCH_LIMIT: return "SOL_ERR_SCRATCH_LIMIT";
     default: return "SOL_ERR_UNKNOWN";
   }
 }
