@@ -32,6 +32,7 @@ sol_status_t check_shape(int B, int H, int N, int d, int block_q, int block_k, b
   if (block_q > 1024 || block_k > 1024) return SOL_ERR_UNSUPPORTED_SHAPE;
   if ((long long)B * H > 0x7fffffLL) return SOL_ERR_UNSUPPORTED_SHAPE;
   if (sol::ceil_div(N, block_k) > 65535 || sol::ceil_div(N, block_q) > 65535) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H * sol::ceil_div(N, block_q) > 0x7fffffffLL) return SOL_ERR_UNSUPPORTED_SHAPE;   // work items are counted in int32
   if (fused && (block_q != block_k || (block_q != 64 && block_q != 128))) return SOL_ERR_UNSUPPORTED_SHAPE;
   return SOL_OK;
 }

@@ -44,26 +44,29 @@ constexpr int kHalf = 64;                        // key columns per softmax warp
 constexpr int kThreads = 384;
 constexpr int kTileBytes = kBlk * kD * 2;        // 32 KB: one K-like or V-like tile
 constexpr int kHalfBytes = kTileBytes / 2;       // 16 KB: 64 channels x 128 rows (one TMA box)
-constexpr int kStages = 5;                       // ring of K/V tiles
+constexpr int kStages = 4;                       // ring of K/V tiles
+constexpr int kGroup = 32;                       // pooled keys scored per router step (one per lane)
 constexpr int kRecords = 4;                      // ring of routing records
 constexpr int kTmemCols = 512;
 constexpr int kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units
-constexpr int kStaggerCycles = 500;              // head start of softmax group 0 over group 1, per work item
+constexpr int kStaggerCycles = 0;                // head start of softmax group 0 over group 1, per work item
 constexpr int kPolyEvery = 0;                    // every n-th exp2 runs on the FMA pipe instead of MUFU (0: none)
 
 constexpr uint8_t kRecFirst = 1, kRecLast = 2, kRecApprox = 4;
 
-struct Record {
+struct alignas(16) Record {
+  float bias[kBlk];             // approximate-tile column bias: log2(n_j) / (scale * log2 e), or -inf
   int32_t work;                 // bh * Nq + i, or -1: no more work
   int16_t chunk;
   uint8_t flags;
   uint8_t n_sel;
   uint8_t sel[kBlk];            // offsets (within the chunk) of the routed blocks
-  float bias[kBlk];             // approximate-tile column bias: log2(n_j), or -inf
 };
 
 struct Shared {
+  float kc_stage[2][kGroup * kD];   // router: fp32 pooled keys of the group being scored / the next one
+  float qbar_s[kD];                 // router: pooled query of the current work item
   Record rec[kRecords];
   float2 ml[2][kBlk];           // (m_h, l_h) exchange between the softmax warpgroups
   uint64_t rec_full[kRecords], rec_empty[kRecords];
@@ -71,6 +74,7 @@ struct Shared {
   uint64_t q_full, q_empty;
   uint64_t s_full[2], p_full[2][2], pv_done[2];   // indexed by score buffer (and warpgroup)
   uint64_t x_full, x_done;      // rendezvous of the two softmax warpgroups at the end of a work item
+  uint64_t kc_full[2];          // router staging buffers filled
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -230,9 +234,10 @@ __device__ __forceinline__ Event next_event(Shared& sm, Cursor& c, long long* wa
 // router: one warp
 __device__ void router_role(Shared& sm, const Params& p, int lane) {
   const unsigned full = 0xffffffffu;
-  uint32_t n_rec = 0;
+  uint32_t n_rec = 0, n_copy = 0, n_use = 0;   // records written; staging copies issued / consumed
   const int n_chunks = ceil_div(p.Nk, kBlk);
   const int mask_words = ceil_div(p.Nk, 32);
+  const float inv_sl2 = 1.f / (p.scale * 1.4426950408889634f);   // biases are stored in raw-score units
   bool alive = true;
   PROF_DECL
   while (alive) {
@@ -241,14 +246,32 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
     w = __shfl_sync(full, w, 0);
     if (w >= p.total_work) break;
     const int bh = w / p.Nq, i = w - bh * p.Nq;
-    float4 qb = make_float4(0.f, 0.f, 0.f, 0.f);
+    // the pooled query of this work item goes to shared memory (one 16-byte piece per lane)
     float tau_i = 0.f;
     if (p.mode != SOL_MODE_DENSE) {
-      qb = *reinterpret_cast<const float4*>(p.qbar + ((size_t)bh * p.Nq + i) * kD + lane * 4);
+      __syncwarp();
+      reinterpret_cast<float4*>(sm.qbar_s)[lane] =
+          __ldg(reinterpret_cast<const float4*>(p.qbar + ((size_t)bh * p.Nq + i) * kD) + lane);
       tau_i = p.tau[(size_t)bh * p.Nq + i];
+      __syncwarp();
     }
     const float* kc_head = p.kc + (size_t)bh * p.Nk * kD;
     int count = 0;
+    // Bulk-copy one group of 32 pooled keys (16 KB, contiguous in memory) into a staging buffer;
+    // the copy of group n+1 is in flight while group n is scored.
+    auto stage_group = [&](int jb) {
+      if (p.mode == SOL_MODE_DENSE || jb >= p.Nk) return;
+      __syncwarp();                                  // every lane is done reading this buffer
+      if (lane == 0) {
+        const uint32_t buf = n_copy & 1;
+        const uint32_t bytes = (uint32_t)min(kGroup, p.Nk - jb) * kD * 4;
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(&sm.kc_full[buf], bytes);
+        bulk_load_1d(sm.kc_stage[buf], kc_head + (size_t)jb * kD, bytes, &sm.kc_full[buf]);
+      }
+      ++n_copy;
+    };
+    stage_group(0);
     for (int t = 0; t < n_chunks; ++t) {
       Record& rec = sm.rec[n_rec % kRecords];
       if (!WAIT(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, 0)) {   // prof 0: record ring full
@@ -267,39 +290,40 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
         if (p.mode == SOL_MODE_DENSE) {
           sel = j < p.Nk;
         } else {
-          // lane owns channels 4*lane..4*lane+3.  Eight pooled keys at a time: partial dot
-          // products, a transposing butterfly over lane bits 0-2 and two plain exchanges leave the
-          // dot product of key (8*sub + (lane & 7)) in every lane; lanes 8*sub..8*sub+7 keep it.
+          // lane l scores pooled key jbase + l against the staged rows.  Lane l starts at 16-byte
+          // piece l of its row and of the query and walks round, so that the 32 lanes hit 32
+          // different shared-memory bank groups although the rows are 512 bytes apart.
           float dot = 0.f;
-#pragma unroll 1
-          for (int sub = 0; sub < 4; ++sub) {
-            float v[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-              const int jr = min(jbase + sub * 8 + r, p.Nk - 1);
-              const float4 kk = __ldg(reinterpret_cast<const float4*>(kc_head + (size_t)jr * kD + lane * 4));
-              v[r] = fmaf(qb.x, kk.x, fmaf(qb.y, kk.y, fmaf(qb.z, kk.z, qb.w * kk.w)));
+          if (jbase < p.Nk) {
+            const uint32_t buf = n_use & 1;
+            if (!WAIT(&sm.kc_full[buf], (n_use >> 1) & 1, 1)) {                         // prof 1: pooled keys not staged
+              if (lane == 0) flag_abort(sm, p, 102);
+              alive = false;
+              break;
             }
+            ++n_use;
+            stage_group(jbase + kGroup);              // next group of this work item, if any
+            const float4* row = reinterpret_cast<const float4*>(sm.kc_stage[buf] + lane * kD);
+            const float4* qv = reinterpret_cast<const float4*>(sm.qbar_s);
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int off = 4; off >= 1; off >>= 1) {
-#pragma unroll
-              for (int r = 0; r < off; ++r) {
-                const bool up = (lane & off) != 0;
-                const float send = up ? v[r] : v[r + off];
-                const float keep = up ? v[r + off] : v[r];
-                v[r] = keep + __shfl_xor_sync(full, send, off);
-              }
+            for (int c = 0; c < kD / 4; ++c) {
+              const int piece = (c + lane) & (kD / 4 - 1);
+              const float4 kk = row[piece];
+              const float4 qq = qv[piece];
+              a0 = fmaf(qq.x, kk.x, a0);
+              a1 = fmaf(qq.y, kk.y, a1);
+              a2 = fmaf(qq.z, kk.z, a2);
+              a3 = fmaf(qq.w, kk.w, a3);
             }
-            v[0] += __shfl_xor_sync(full, v[0], 8);
-            v[0] += __shfl_xor_sync(full, v[0], 16);
-            if ((lane >> 3) == sub) dot = v[0];
+            dot = (a0 + a1) + (a2 + a3);
           }
           sel = (j < p.Nk) && (p.scale * dot > tau_i);
         }
         const unsigned m = __ballot_sync(full, sel);
         const bool valid = j < p.Nk;
         any_unselected |= (valid && !sel);
-        rec.bias[g * 32 + lane] = (valid && !sel) ? log2f((float)min(kBlk, p.N - j * kBlk)) : -INFINITY;
+        rec.bias[g * 32 + lane] = (valid && !sel) ? log2f((float)min(kBlk, p.N - j * kBlk)) * inv_sl2 : -INFINITY;
         if (sel) rec.sel[n_sel + __popc(m & ((1u << lane) - 1u))] = (uint8_t)(g * 32 + lane);
         n_sel += __popc(m);
         if (p.mask_out && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
@@ -495,7 +519,6 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
   const uint32_t t_o_other = lane_base + kTmemO + (1 - h) * kD;
   const int row = warp_in_group * 32 + lane;
   const float sl2 = p.scale * 1.4426950408889634f;
-  const float inv_sl2 = 1.f / sl2;
   uint32_t g = 0, n_merge = 0;
   bool stagger = true;
   float m_used = -INFINITY, l = 0.f;
@@ -538,11 +561,20 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       if (general) {
         // bring the rare tiles (approximate chunk, ragged last block) to the common form
         // logit = sl2 * x by folding the column bias into x; -inf marks masked columns
+        if (approx) {
+          const float4* bias4 = reinterpret_cast<const float4*>(&ev.rec->bias[h * kHalf]);
 #pragma unroll
-        for (int c = 0; c < kHalf; ++c) {
-          const float x = __uint_as_float(sr[c]);
-          const int col = h * kHalf + c;
-          sr[c] = __float_as_uint(approx ? fmaf(ev.rec->bias[col], inv_sl2, x) : (col < cols_valid ? x : -INFINITY));
+          for (int c = 0; c < kHalf / 4; ++c) {
+            const float4 bb = bias4[c];
+            sr[4 * c] = __float_as_uint(__uint_as_float(sr[4 * c]) + bb.x);
+            sr[4 * c + 1] = __float_as_uint(__uint_as_float(sr[4 * c + 1]) + bb.y);
+            sr[4 * c + 2] = __float_as_uint(__uint_as_float(sr[4 * c + 2]) + bb.z);
+            sr[4 * c + 3] = __float_as_uint(__uint_as_float(sr[4 * c + 3]) + bb.w);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < kHalf; ++c)
+            if (h * kHalf + c >= cols_valid) sr[c] = __float_as_uint(-INFINITY);
         }
       }
       float mx;
@@ -607,6 +639,9 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       tc_fence_before();
       mbar_arrive(&sm.p_full[h][b]);
       PROF_ADD(9)                                                                      // prof 9: whole tile
+#ifdef SOL_PROFILE
+      if (approx) { prof.v[10] += clock64() - prof_t0; ++prof.v[0]; }                  // prof 10 / 0: approximate tiles: cycles / count
+#endif
       PROF_COUNT(5);                                                                    // prof 5: tiles
       ++g;
       continue;
@@ -616,6 +651,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     const int bh = ev.work / p.Nq, i = ev.work - bh * p.Nq;
     const int q_rows = min(kBlk, p.N - i * kBlk);
     __nv_bfloat16* orow = p.out + ((size_t)bh * p.N + (size_t)i * kBlk + row) * kD + h * kHalf;
+    PROF_T0
     if (!ev.first) {
       // the last P V of the item (one commit covers both halves)
       if (!WAIT(&sm.pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, 3)) { flag_abort(sm, p, 403); break; }   // prof 3
@@ -669,6 +705,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     }
     m_used = -INFINITY;
     l = 0.f;
+    PROF_ADD(2)                                                                        // prof 2: whole epilogue
   }
   if (lane == 0 && warp_in_group == 0 && h == 0) PROF_FLUSH(3);
 }
@@ -697,6 +734,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       mbar_init(&sm.p_full[1][b], 128);
     }
     mbar_init(&sm.x_full, 256); mbar_init(&sm.x_done, 256);
+    mbar_init(&sm.kc_full[0], 1); mbar_init(&sm.kc_full[1], 1);
     fence_mbar_init();
   }
   if (warp == 9 && lane == 0) {
