@@ -241,3 +241,32 @@ def test_bound_entry_points_and_host_path():
         refd = orc.dense_attention(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
                                    synth.widen(vb[0, h], np.float64))
         assert (np.abs(hp.dev_to_f64(dense)[0, h] - refd) <= hp.out_bound(refd)).all()
+
+
+@pytest.mark.parametrize("impl", IMPLS_128)
+@pytest.mark.parametrize("jump", [3.0, 6.0])
+def test_reference_maximum_jumps(impl, jump):
+    """Late key blocks whose logits tower over everything before them: the running maximum has to
+    be raised (moderately: before the next tile; hugely: the tile is recomputed) without losing
+    the earlier blocks' exact contribution.  All queries share a direction u; the keys of the last
+    third of the sequence get multiples of u, growing block by block."""
+    B, H, N, d = 1, 2, 1536, 128
+    rng = np.random.default_rng(99)
+    x = rng.standard_normal((3, B, H, N, d)).astype(np.float32)
+    u = rng.standard_normal(d).astype(np.float32)
+    x[0] += u                                                   # q . u is about |u|^2 = 128
+    for j, blk in enumerate(range(8, 12)):                      # blocks 8..11 of 12
+        x[1][:, :, blk * 128:(blk + 1) * 128] += (j + 1) * jump * u   # logits rise by ~ jump * 11.3 nats per block
+    bits = [synth.f32_to_bf16_bits(x[i]) for i in range(3)]
+    for beta, mode, name in [(0.0, sb.SOL_MODE_DENSE, "sol"), (-0.2, sb.SOL_MODE_SOL, "sol"), (0.8, sb.SOL_MODE_SOL, "sol")]:
+        if mode == sb.SOL_MODE_DENSE:
+            qb, kb, vb = bits
+            q, k, v = (hp.to_dev(t) for t in bits)
+            out, _, _, _ = hp.run_gpu(q, k, v, 128, 0.0, mode=mode, impl=_impl(impl), want_mask=False)
+            o = hp.dev_to_f64(out)
+            for h in range(H):
+                ref = orc.dense_attention(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                                          synth.widen(vb[0, h], np.float64))
+                assert (np.abs(o[0, h] - ref) <= hp.out_bound(ref)).all()
+        else:
+            _check_all_heads(bits, 128, beta, _impl(impl))
