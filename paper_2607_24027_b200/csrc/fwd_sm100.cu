@@ -94,7 +94,7 @@ struct Params {
 __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int where) {
   sm.abort_flag = 1;
   atomicExch(p.status + kStatusDevice, (int)SOL_ERR_DEVICE_TIMEOUT);
-  atomicExch(p.status + kStatusDetail, where);
+  atomicCAS(p.status + kStatusDetail, 0, where);     // keep the first place that gave up
 }
 
 // 2^x for x <= ~8 without the MUFU unit: round-to-nearest split x = n + f, f in [-0.5, 0.5],
