@@ -51,7 +51,6 @@ constexpr int kTmemCols = 512;
 constexpr int kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units
 constexpr int kStaggerCycles = 0;                // head start of softmax group 0 over group 1, per work item
-constexpr int kPolyEvery = 0;                    // every n-th exp2 runs on the FMA pipe instead of MUFU (0: none)
 
 constexpr uint8_t kRecFirst = 1, kRecLast = 2, kRecApprox = 4;
 
@@ -97,18 +96,6 @@ __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int wher
   atomicCAS(p.status + kStatusDetail, 0, where);     // keep the first place that gave up
 }
 
-// 2^x for x <= ~8 without the MUFU unit: round-to-nearest split x = n + f, f in [-0.5, 0.5],
-// cubic minimax polynomial for 2^f (max relative error 7.5e-5, far below bf16 resolution), and n
-// added straight into the exponent field.
-__device__ __forceinline__ float exp2_poly(float x) {
-  x = fmaxf(x, -126.f);
-  const float magic = 12582912.f;               // 1.5 * 2^23: the low mantissa bits of x + magic hold n
-  const float r = x + magic;
-  const float f = x - (r - magic);
-  const float pz = fmaf(fmaf(fmaf(0.055171460f, f, 0.24261086f), f, 0.69326097f), f, 0.99992812f);
-  return __int_as_float(__float_as_int(pz) + (__float_as_int(r) << 23));
-}
-
 // Optional per-role cycle accounting (build with -DSOL_PROFILE): how long each role spends in
 // each kind of wait.  Slot meaning is listed next to every use; read back with
 // sol_attn_debug_profile().
@@ -139,6 +126,10 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_COUNT(slot) (++prof.v[slot])
 #define PROF_FLUSH(role) prof.flush(role)
 #define PROF_ACC(slot) (&prof.v[slot])
+// timeline of a few tiles of CTA 0: [tile][event] = clock64()
+constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 12;
+__device__ long long g_trace[kTraceTiles * kTraceEvents];
+#define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
 #define PROF_T0 const long long prof_t0 = clock64();
 #define PROF_ADD(slot) prof.v[slot] += clock64() - prof_t0;
 #else
@@ -147,6 +138,7 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_COUNT(slot)
 #define PROF_FLUSH(role)
 #define PROF_ACC(slot) nullptr
+#define TRACE(tile, evt)
 #define PROF_T0
 #define PROF_ADD(slot)
 #endif
@@ -450,6 +442,7 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
     // the previous user of this score buffer was tile g-2: its P V must have read P out of it
     if (g >= 2 && !WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }   // prof 3: score buffer busy
     tc_fence_after();
+    TRACE(g, 0);
     {
       PROF_T0
       const uint32_t k_lo = kv_lo + slot * (kTileBytes >> 4);
@@ -463,6 +456,7 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
       mma_commit(&sm.s_full[b]);
       PROF_ADD(6)                                                                      // prof 6: issuing Q K^T
     }
+    TRACE(g, 1);
     ++g;
     slot += 2;                                    // K tiles sit at every other ring position
     if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
@@ -487,11 +481,13 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
     if (ev.type != kEvTile) continue;
     const uint32_t b = g & 1;
     if (!mbar_wait(&sm.kv_full[slot], slot_parity, &sm.abort_flag)) { ok = false; break; }
+    TRACE(g, 2);
     const uint32_t v_lo = kv_lo + slot * (kTileBytes >> 4);
     const uint32_t acc_first = ev.first ? 0u : 1u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag)) { ok = false; break; }
+      TRACE(g, 3 + h);
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < kHalf / 16; ++ks) {
@@ -502,6 +498,7 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
     if (!ok) break;
     mma_commit(&sm.kv_empty[slot]);
     mma_commit(&sm.pv_done[b]);
+    TRACE(g, 5);
     ++g;
     slot += 2;
     if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
@@ -551,6 +548,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       const bool general = approx || cols_valid < kBlk;
       if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
       tc_fence_after();
+      if (row == 0) TRACE(g, 6 + 3 * h);
       // ---- this group's half row of S (64 fp32) into registers with one wait
       uint32_t sr[kHalf];
       PROF_T0
@@ -612,32 +610,34 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         l *= f;
         m_used = m_new;
       }
-      // ---- P = exp2(sl2 * S - m): most elements on the MUFU unit, every kPolyEvery-th one as a
-      //      polynomial on the FMA pipe; row sum; P (bf16) back to TMEM over the start of the half
+      // ---- P = exp2(sl2 * S - m) (scaling and row sum as packed fp32 pairs); P (bf16) back to
+      //      TMEM over the start of the half
       {
         const float nm = (m_used == -INFINITY) ? 0.f : -m_used;   // a half that has seen nothing yet: all P = 0
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        const uint64_t sl2_2 = pack2(sl2, sl2), nm2 = pack2(nm, nm);
+        uint64_t s_a = pack2(0.f, 0.f), s_b = pack2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < kHalf; c += 4) {
-          float e[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const float x = fmaf(__uint_as_float(sr[c + u]), sl2, nm);
-            e[u] = (kPolyEvery > 0 && ((c + u) % kPolyEvery) == kPolyEvery - 1) ? exp2_poly(x) : ex2(x);
-          }
-          sum0 += e[0]; sum1 += e[1]; sum2 += e[2]; sum3 += e[3];
-          __nv_bfloat162 lo = __floats2bfloat162_rn(e[0], e[1]);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(e[2], e[3]);
+          float xa, xb, xc, xd;
+          unpack2(fma2(pack2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sl2_2, nm2), xa, xb);
+          unpack2(fma2(pack2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sl2_2, nm2), xc, xd);
+          const float e0 = ex2(xa), e1 = ex2(xb), e2 = ex2(xc), e3 = ex2(xd);
+          s_a = add2(s_a, pack2(e0, e1));
+          s_b = add2(s_b, pack2(e2, e3));
+          __nv_bfloat162 lo = __floats2bfloat162_rn(e0, e1);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(e2, e3);
           sr[c / 2] = *reinterpret_cast<uint32_t*>(&lo);
           sr[c / 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
         }
-        l += (sum0 + sum1) + (sum2 + sum3);
+        { float t0, t1; unpack2(add2(s_a, s_b), t0, t1); l += t0 + t1; }
         tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
       }
       PROF_ADD(8)                                                                      // prof 8: load + arithmetic
+      if (row == 0) TRACE(g, 7 + 3 * h);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&sm.p_full[h][b]);
+      if (row == 0) TRACE(g, 8 + 3 * h);
       PROF_ADD(9)                                                                      // prof 9: whole tile
 #ifdef SOL_PROFILE
       if (approx) { prof.v[10] += clock64() - prof_t0; ++prof.v[0]; }                  // prof 10 / 0: approximate tiles: cycles / count
@@ -772,6 +772,9 @@ extern "C" int sol_attn_debug_profile(long long* host_out, int n_values) {
   const size_t total = sizeof(long long) * sol::kProfCtas * sol::kProfRoles * sol::kProfSlots;
   const size_t want = sizeof(long long) * (size_t)n_values;
   return (int)cudaMemcpyFromSymbol(host_out, sol::g_prof, want < total ? want : total);
+}
+extern "C" int sol_attn_debug_trace(long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, sol::g_trace, sizeof(long long) * sol::kTraceTiles * sol::kTraceEvents);
 }
 namespace sol {
 #endif
