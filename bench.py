@@ -180,6 +180,35 @@ def run_reference(args, wl, beta):
     print(json.dumps(line), flush=True)
 
 
+def run_ablation(sb, to_dev, name="image"):
+    """rel-L2 / cosine of the output against dense attention (all on the GPU, same kernel in dense
+    mode), for Sol-Attn and for keep-or-drop sparsity under the same routing; per-query-block
+    density percentiles from the counts output."""
+    import torch
+    wl = WORKLOADS[name]
+    qb, kb, vb = synth.generate(wl)
+    q, k, v = to_dev(qb), to_dev(kb), to_dev(vb)
+    B, H, N, d = q.shape
+    ws = sb.make_workspace(B, H, N, d, wl.block, wl.block)
+    dense, out = torch.empty_like(q), torch.empty_like(q)
+    sb.sol_attn_forward_ex(q, k, v, dense, ws, wl.block, wl.block, mode=sb.SOL_MODE_DENSE)
+    ref = dense.float()
+    rows = []
+    for rho, beta in sorted(load_betas()[name].items()):
+        rec = {"target_density": rho, "beta": beta}
+        for label, mode in (("sol", sb.SOL_MODE_SOL), ("exact_only", sb.SOL_MODE_EXACT_ONLY)):
+            sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=beta, mode=mode)
+            o = out.float()
+            rec[label + "_rel_l2"] = float((o - ref).norm() / ref.norm())
+            rec[label + "_cosine"] = float(torch.nn.functional.cosine_similarity(o.flatten(), ref.flatten(), dim=0))
+        dens = ws.counts.float().flatten() / wl.n_blocks
+        rec["density"] = float(dens.mean())
+        rec["per_block_density_p10_p50_p90"] = [float(x) for x in torch.quantile(dens, torch.tensor([0.1, 0.5, 0.9], device=dens.device))]
+        rows.append(rec)
+    torch.cuda.synchronize()
+    return {"workload": name, "rows": rows}
+
+
 # ------------------------------------------------------------------------------------------ GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -335,6 +364,13 @@ def main():
                           "speedup_vs_dense": ms_dense / ms_f, "one_over_density": 1.0 / dens})
         check_status()
 
+    # ---- accuracy ablation on the image workload (small): error against dense attention of the
+    #      full method vs keep-or-drop block-sparse attention under the SAME mask, and the spread of
+    #      per-query-block densities (the counts output)
+    ablation = None
+    if not args.no_sweep and world == 1:
+        ablation = run_ablation(sb, to_dev)
+
     if world > 1:
         dist.barrier()
     if rank != 0:
@@ -378,6 +414,7 @@ def main():
                  "pre_attention_ms": ms_pool},
         "cpu_baseline": cpu,
         "sweep": sweep,
+        "ablation": ablation,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

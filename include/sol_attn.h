@@ -58,6 +58,13 @@ enum {
   SOL_MODE_EXACT_ONLY = 2   /* Eq. (2): routed blocks exact, unselected blocks dropped         */
 };
 
+/* how sigma_i of Eq. (4) is estimated in the pre-attention pass */
+enum {
+  SOL_EST_MOMENTS  = 0,   /* exact: full second moment of the pooled keys, Eq. (5)                */
+  SOL_EST_DIAGONAL = 1    /* diagonal of the pooled-key covariance only (appendix, diagonal
+                             threshold estimator): O(d) per query block                         */
+};
+
 /* which implementation of the fused kernel runs */
 enum {
   SOL_IMPL_AUTO     = 0,  /* tcgen05 kernel when the shape allows it, else the mma.sync one    */
@@ -132,6 +139,13 @@ typedef struct {
                                                    S_i; NULL in production (the proxy map is
                                                    never written to memory otherwise)           */
   sol_stream_t stream;
+  int32_t estimator;                            /* SOL_EST_* (0 = Eq. 5 moments)                */
+  const uint8_t* forced_blocks;                 /* device uint8 [ceil(N/block_k)] or NULL: key
+                                                   blocks with a nonzero entry are always routed
+                                                   to the exact branch, whatever their proxy score
+                                                   (text / sink key-value tokens kept exact, as in
+                                                   the paper's MMDiT integrations); shared by all
+                                                   batches and heads; counts include them         */
 } sol_attn_args;
 sol_status_t sol_attn_forward_ex(const sol_attn_args* args /* host */);
 

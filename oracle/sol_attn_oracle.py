@@ -317,15 +317,27 @@ class SolAttnResult:
 
 
 def routing(q, k, v, block_q: int, block_k: int, beta: float,
-            scale: Optional[float] = None, dtype=np.float64):
-    """Pre-attention step only: pooled tensors, proxy rows, thresholds and the block mask."""
+            scale: Optional[float] = None, dtype=np.float64, estimator: str = "direct", forced=None):
+    """Pre-attention step only: pooled tensors, proxy rows, thresholds and the block mask.
+
+    ``estimator``: "direct" (row statistics of the proxy row, Eq. 4 -- equal to the moment form of
+    Eq. 5) or "diagonal" (Eq. appendix_diagonal_threshold).  ``forced``: optional bool [N_k]; those
+    key blocks are put into every S_i regardless of their score (text / sink key-value tokens that
+    the paper's model integrations keep in the exact branch)."""
     q = np.asarray(q, dtype=dtype)
     d = q.shape[1]
     s = default_scale(d) if scale is None else scale
     qbar, kc, vc, _ = pool(q, k, v, block_q, block_k, dtype=dtype)
     s_hat = proxy_scores(qbar, kc, s)
-    mu, sigma, tau = threshold_direct(s_hat, beta)
+    if estimator == "direct":
+        mu, sigma, tau = threshold_direct(s_hat, beta)
+    elif estimator == "diagonal":
+        mu, sigma, tau = threshold_diagonal(qbar, kc, beta, s)
+    else:
+        raise ValueError(estimator)
     mask = select_blocks(s_hat, tau)
+    if forced is not None:
+        mask = mask | np.asarray(forced, dtype=bool)[None, :]
     return SolAttnResult(out=None, mask=mask, counts=mask.sum(axis=1), s_hat=s_hat, mu=mu,
                          sigma=sigma, tau=tau, qbar=qbar, kc=kc, vc=vc)
 
@@ -333,9 +345,11 @@ def routing(q, k, v, block_q: int, block_k: int, beta: float,
 def sol_attn_forward(q, k, v, block_q: int, block_k: int, beta: float,
                      scale: Optional[float] = None, chunk: int = 16, dtype=np.float64,
                      q_tiles: Optional[Sequence[int]] = None, mask_override=None,
-                     exact_only: bool = False) -> SolAttnResult:
+                     exact_only: bool = False, estimator: str = "direct", forced=None) -> SolAttnResult:
     """The hot path for one head: pool -> proxy row -> tau_i -> Algorithm 1."""
-    r = routing(q, k, v, block_q, block_k, beta, scale=scale, dtype=dtype)
+    r = routing(q, k, v, block_q, block_k, beta, scale=scale, dtype=dtype, estimator=estimator, forced=forced)
+    if forced is not None and mask_override is None:
+        mask_override = r.mask          # Algorithm 1 run under the routed-or-forced mask
     out, mask = sol_attn_streaming(q, k, v, r.kc, r.vc, r.tau, block_q, block_k, chunk=chunk,
                                    scale=scale, dtype=dtype, q_tiles=q_tiles,
                                    mask_override=mask_override, exact_only=exact_only)

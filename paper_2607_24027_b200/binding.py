@@ -27,6 +27,7 @@ SOL_ERR_SCRATCH_LIMIT = -7
 
 SOL_MODE_SOL, SOL_MODE_DENSE, SOL_MODE_EXACT_ONLY = 0, 1, 2
 SOL_IMPL_AUTO, SOL_IMPL_TCGEN05, SOL_IMPL_MMA_SYNC = 0, 1, 2
+SOL_EST_MOMENTS, SOL_EST_DIAGONAL = 0, 1
 
 EXPORTS = [
     "sol_attn_status_string", "sol_attn_workspace_bytes", "sol_attn_workspace_view",
@@ -59,6 +60,7 @@ class _Args(ctypes.Structure):
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("counts", ctypes.c_void_p), ("mask_out", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
+        ("estimator", ctypes.c_int32), ("forced_blocks", ctypes.c_void_p),
     ]
 
 
@@ -220,14 +222,14 @@ def sol_attn_dense(q, k, v, out, stream=None):
 
 def sol_attn_forward_ex(q, k, v, out, ws: Workspace, block_q, block_k, threshold=0.0, scale=0.0,
                         mode=SOL_MODE_SOL, impl=SOL_IMPL_AUTO, skip_pool=False, tau_override=None,
-                        counts=None, mask_out=None, stream=None):
+                        counts=None, mask_out=None, stream=None, estimator=SOL_EST_MOMENTS, forced_blocks=None):
     B, H, N, d = _dims(q)
     a = _Args(q=_ptr(q), k=_ptr(k), v=_ptr(v), out=_ptr(out), B=B, H=H, N=N, d=d,
               block_q=block_q, block_k=block_k, threshold=float(threshold), scale=float(scale),
               mode=mode, impl=impl, skip_pool=int(skip_pool), tau_override=_ptr(tau_override),
               workspace=ws.buf.data_ptr(), workspace_bytes=ws.buf.numel(),
               counts=_ptr(counts if counts is not None else ws.counts), mask_out=_ptr(mask_out),
-              stream=_stream(stream))
+              stream=_stream(stream), estimator=int(estimator), forced_blocks=_ptr(forced_blocks))
     _check(lib().sol_attn_forward_ex(ctypes.byref(a)), "sol_attn_forward_ex")
 
 

@@ -27,6 +27,8 @@ struct Problem {
   float scale;       // logit scale
   float beta;        // standardized cutoff of Eq. (4)
   int mode;          // SOL_MODE_*
+  int estimator;     // SOL_EST_*: how sigma_i is obtained
+  const uint8_t* forced;   // device [Nk] or null: key blocks that always go to the exact branch
 };
 
 // Byte offsets into the workspace (all multiples of 1024).

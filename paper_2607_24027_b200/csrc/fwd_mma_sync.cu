@@ -76,7 +76,8 @@ __global__ void __launch_bounds__(BLK * 2)
 fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ out,
                     WsPtrs ws, const float* __restrict__ tau, int32_t* __restrict__ counts,
-                    uint32_t* __restrict__ mask_out, int N, int Nq, int Nk, float scale, int mode) {
+                    uint32_t* __restrict__ mask_out, const uint8_t* __restrict__ forced, int N, int Nq, int Nk,
+                    float scale, int mode) {
   constexpr int THREADS = BLK * 2;
   constexpr int WARPS = THREADS / 32;
   constexpr int NT = BLK / 8;                   // score n-tiles (8 key columns each)
@@ -216,6 +217,7 @@ fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
           sel = scale * dot > tau_i;
+          if (forced && forced[j]) sel = true;
         }
         if (!sel) bias = log2f((float)min(BLK, N - j * BLK));
       }
@@ -283,7 +285,7 @@ cudaError_t launch_impl(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.Nq, p.BH);
-  fwd_mma_sync_kernel<D, BLK><<<grid, BLK * 2, smem, stream>>>(q, k, v, out, ws, tau, counts, mask_out,
+  fwd_mma_sync_kernel<D, BLK><<<grid, BLK * 2, smem, stream>>>(q, k, v, out, ws, tau, counts, mask_out, p.forced,
                                                                 p.N, p.Nq, p.Nk, p.scale, p.mode);
   return cudaGetLastError();
 }

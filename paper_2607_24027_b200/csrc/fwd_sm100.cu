@@ -88,6 +88,7 @@ struct Params {
   int32_t* status;              // workspace status words
   int N, Nq, Nk, total_work, mode;
   float scale;
+  const uint8_t* forced;        // [Nk] or null: key blocks always routed to the exact branch
 };
 
 __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int where) {
@@ -311,6 +312,7 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
             dot = (a0 + a1) + (a2 + a3);
           }
           sel = (j < p.Nk) && (p.scale * dot > tau_i);
+          if (p.forced && j < p.Nk && p.forced[j]) sel = true;
         }
         const unsigned m = __ballot_sync(full, sel);
         const bool valid = j < p.Nk;
@@ -792,7 +794,7 @@ cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __n
   Params prm{};
   prm.qbar = ws.qbar; prm.kc = ws.kc; prm.tau = tau; prm.out = out; prm.counts = counts; prm.mask_out = mask_out;
   prm.status = ws.status; prm.N = p.N; prm.Nq = p.Nq; prm.Nk = p.Nk; prm.total_work = p.BH * p.Nq;
-  prm.mode = p.mode; prm.scale = p.scale;
+  prm.mode = p.mode; prm.scale = p.scale; prm.forced = p.forced;
 
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -257,8 +257,76 @@ cudaError_t launch_pool(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
   return cudaGetLastError();
 }
 
+// Diagonal estimator (appendix, Eq. appendix_diagonal_threshold): only the per-channel variance of
+// the pooled keys is kept, v_K = mean_j KC_j o KC_j - m_K o m_K (computed in centred form), and
+// sigma_i^2 = s^2 (Qbar_i o Qbar_i) . v_K.  One CTA per (batch, head) writes m_K and v_K (v_K goes
+// to the first D floats of the head's second-moment area).
+template <int D>
+__global__ void __launch_bounds__(4 * D) key_diag_kernel(WsPtrs ws, int Nk) {
+  __shared__ float part[4][D];
+  __shared__ float mean_s[D];
+  const int bh = blockIdx.x, c = threadIdx.x % D, grp = threadIdx.x / D;
+  const float* kc = ws.kc + (size_t)bh * Nk * D;
+  float s = 0.f;
+  for (int j = grp; j < Nk; j += 4) s += kc[(size_t)j * D + c];
+  part[grp][c] = s;
+  __syncthreads();
+  if (grp == 0) mean_s[c] = ((part[0][c] + part[1][c]) + (part[2][c] + part[3][c])) / (float)Nk;
+  __syncthreads();
+  const float m = mean_s[c];
+  float v = 0.f;
+  for (int j = grp; j < Nk; j += 4) {
+    const float x = kc[(size_t)j * D + c] - m;
+    v = fmaf(x, x, v);
+  }
+  __syncthreads();
+  part[grp][c] = v;
+  __syncthreads();
+  if (grp == 0) {
+    ws.mk[(size_t)bh * D + c] = m;
+    ws.covk[(size_t)bh * D * D + c] = ((part[0][c] + part[1][c]) + (part[2][c] + part[3][c])) / (float)Nk;
+  }
+}
+
+// One warp per query block: mu_i, sigma_i (diagonal form), tau_i.
+template <int D>
+__global__ void __launch_bounds__(256) tau_diag_kernel(WsPtrs ws, int Nq, float scale, float beta) {
+  const int bh = blockIdx.y;
+  const int i = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+  if (i >= Nq) return;
+  const float* qb = ws.qbar + ((size_t)bh * Nq + i) * D;
+  const float* mk = ws.mk + (size_t)bh * D;
+  const float* vk = ws.covk + (size_t)bh * D * D;
+  float quad = 0.f, dotm = 0.f;
+#pragma unroll
+  for (int c = lane; c < D; c += 32) {
+    const float qv = qb[c];
+    quad = fmaf(qv * qv, vk[c], quad);
+    dotm = fmaf(qv, mk[c], dotm);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    quad += __shfl_xor_sync(0xffffffffu, quad, o);
+    dotm += __shfl_xor_sync(0xffffffffu, dotm, o);
+  }
+  if (lane == 0) {
+    const float mu = scale * dotm;
+    const float sigma = scale * sqrtf(fmaxf(quad, 0.f));
+    const size_t o = (size_t)bh * Nq + i;
+    ws.mu[o] = mu;
+    ws.sigma[o] = sigma;
+    ws.tau[o] = isinf(beta) ? beta : fmaf(beta, sigma, mu);
+  }
+}
+
 template <int D>
 static cudaError_t thresholds_impl(const Problem& p, const WsPtrs& ws, cudaStream_t stream, int* n_launches) {
+  if (p.estimator == SOL_EST_DIAGONAL) {
+    key_diag_kernel<D><<<p.BH, 4 * D, 0, stream>>>(ws, p.Nk);
+    tau_diag_kernel<D><<<dim3(ceil_div(p.Nq, 8), p.BH), 256, 0, stream>>>(ws, p.Nq, p.scale, p.beta);
+    if (n_launches) *n_launches += 2;
+    return cudaGetLastError();
+  }
   key_mean_kernel<D><<<p.BH, 4 * D, 0, stream>>>(ws, p.Nk);
   key_cov_kernel<D><<<dim3(D / 16, p.BH, kCovSlices), 256, 0, stream>>>(ws, p.Nk);
   const size_t smem = sizeof(float) * (D * D + 64 * (D + 1));

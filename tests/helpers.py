@@ -51,7 +51,7 @@ def unpack_mask(words: torch.Tensor, n_k: int) -> np.ndarray:
 
 
 def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, scale=0.0, want_mask=True,
-            tau_override=None, ws=None):
+            tau_override=None, ws=None, estimator=0, forced=None):
     """Run the fused forward through the C ABI; returns (out, counts, mask or None, ws)."""
     B, H, N, d = q.shape
     if ws is None:
@@ -62,7 +62,8 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
     if want_mask:
         mask_words = torch.zeros(B, H, ws.view.n_q_blocks, sb.mask_words(nk), dtype=torch.int32, device="cuda")
     sb.sol_attn_forward_ex(q, k, v, out, ws, block, block, threshold=beta, scale=scale, mode=mode, impl=impl,
-                           mask_out=mask_words, tau_override=tau_override)
+                           mask_out=mask_words, tau_override=tau_override, estimator=estimator,
+                           forced_blocks=(None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.uint8)).cuda()))
     torch.cuda.synchronize()
     sb.sol_attn_bind_workspace(ws)
     st = sb.sol_attn_read_device_status()
@@ -71,7 +72,8 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
     return out, ws.counts.clone(), mask, ws
 
 
-def check_head(qh, kh, vh, out_h, mask_h, counts_h, block, beta, tiles=None, scale=None, mode="sol"):
+def check_head(qh, kh, vh, out_h, mask_h, counts_h, block, beta, tiles=None, scale=None, mode="sol",
+               estimator="direct", forced=None):
     """Compare one head of GPU results with the oracle.
 
     qh, kh, vh: float64 [L, d] inputs; out_h: float64 [L, d] GPU output; mask_h: [Nq, Nk] bool GPU
@@ -79,10 +81,10 @@ def check_head(qh, kh, vh, out_h, mask_h, counts_h, block, beta, tiles=None, sca
     checked (None = all).  Returns a dict of error statistics; raises on a violation.
     """
     L, d = qh.shape
-    r = orc.routing(qh, kh, vh, block, block, beta, scale=scale)
+    r = orc.routing(qh, kh, vh, block, block, beta, scale=scale, estimator=estimator, forced=forced)
     nq = r.mask.shape[0]
     stats = {"in_band_flips": 0, "blocks": int(r.mask.size)}
-    override = None
+    override = r.mask if forced is not None else None
     if mask_h is not None:
         diff = mask_h != r.mask
         band = np.abs(r.s_hat - r.tau[:, None]) < BAND

@@ -44,11 +44,13 @@ def _small_problem(seed, B, H, N, d, structured=True):
     return bits
 
 
-def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=0.0, tiles=None):
+def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=0.0, tiles=None,
+                     estimator="direct", forced=None):
     qb, kb, vb = bits
     q, k, v = (hp.to_dev(x) for x in bits)
     mode = sb.SOL_MODE_SOL if mode is None else mode
-    out, counts, mask, _ = hp.run_gpu(q, k, v, block, beta, mode=mode, impl=impl, scale=scale)
+    out, counts, mask, _ = hp.run_gpu(q, k, v, block, beta, mode=mode, impl=impl, scale=scale,
+                                      estimator=(1 if estimator == "diagonal" else 0), forced=forced)
     B, H, N, d = q.shape
     out64 = hp.dev_to_f64(out)
     agg = {"in_band_flips": 0, "max_abs": 0.0, "rel_l2": 0.0}
@@ -57,7 +59,8 @@ def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=
             st = hp.check_head(synth.widen(qb[b, h], np.float64), synth.widen(kb[b, h], np.float64),
                                synth.widen(vb[b, h], np.float64), out64[b, h], mask[b, h],
                                counts[b, h].cpu().numpy(), block, beta, tiles=tiles,
-                               scale=(scale if scale > 0 else None), mode=mode_name)
+                               scale=(scale if scale > 0 else None), mode=mode_name, estimator=estimator,
+                               forced=forced)
             agg["in_band_flips"] += st["in_band_flips"]
             agg["max_abs"] = max(agg["max_abs"], st["max_abs"])
             agg["rel_l2"] = max(agg["rel_l2"], st["rel_l2"])
@@ -270,3 +273,41 @@ def test_reference_maximum_jumps(impl, jump):
                 assert (np.abs(o[0, h] - ref) <= hp.out_bound(ref)).all()
         else:
             _check_all_heads(bits, 128, beta, _impl(impl))
+
+
+# ----------------------------------------------------------------------------- beyond the core path
+@pytest.mark.parametrize("impl", IMPLS_128)
+def test_diagonal_threshold_estimator(impl):
+    """Eq. (appendix_diagonal_threshold): sigma from the diagonal of the pooled-key covariance."""
+    bits = _small_problem(21, 1, 3, 2048, 128)
+    agg = _check_all_heads(bits, 128, 0.5, _impl(impl), estimator="diagonal")
+    # the two estimators really differ on these inputs (otherwise the test pins nothing)
+    qb, kb, vb = bits
+    r_full = orc.routing(synth.widen(qb[0, 0], np.float64), synth.widen(kb[0, 0], np.float64),
+                         synth.widen(vb[0, 0], np.float64), 128, 128, 0.5)
+    r_diag = orc.routing(synth.widen(qb[0, 0], np.float64), synth.widen(kb[0, 0], np.float64),
+                         synth.widen(vb[0, 0], np.float64), 128, 128, 0.5, estimator="diagonal")
+    assert np.abs(r_full.tau - r_diag.tau).max() > 1e-3
+    print("diagonal", impl, agg)
+
+
+@pytest.mark.parametrize("impl", IMPLS_128)
+def test_forced_exact_key_blocks(impl):
+    """Key blocks flagged as always-exact (text / sink key-value tokens) enter every S_i."""
+    bits = _small_problem(22, 1, 2, 1500, 128)
+    nk = 12
+    forced = np.zeros(nk, dtype=bool)
+    forced[[0, 5, nk - 1]] = True                     # includes the ragged last block
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out, counts, mask, _ = hp.run_gpu(q, k, v, 128, 0.9, impl=_impl(impl), forced=forced)
+    assert mask[..., forced].all()
+    assert (counts.cpu().numpy() >= 3).all()
+    _check_all_heads(bits, 128, 0.9, _impl(impl), forced=forced)
+    # forcing every block is dense attention
+    allf = np.ones(nk, dtype=bool)
+    out2, counts2, _, _ = hp.run_gpu(q, k, v, 128, 0.9, impl=_impl(impl), forced=allf)
+    assert (counts2.cpu().numpy() == nk).all()
+    for h in range(2):
+        ref = orc.dense_attention(synth.widen(bits[0][0, h], np.float64), synth.widen(bits[1][0, h], np.float64),
+                                  synth.widen(bits[2][0, h], np.float64))
+        assert (np.abs(hp.dev_to_f64(out2)[0, h] - ref) <= hp.out_bound(ref)).all()

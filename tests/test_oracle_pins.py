@@ -349,3 +349,25 @@ def test_p12_hand_worked_example():
     # float32 mode stays within float32 rounding of the same numbers
     r32 = orc.sol_attn_forward(q, k, v, b, b, g["beta"], scale=g["scale"], dtype=np.float32)
     np.testing.assert_allclose(r32.out[:, 0], expect, rtol=2e-6)
+
+
+# ------------------------------------------------------------------ forced-exact blocks, diagonal estimator
+def test_forced_blocks_and_diagonal_routing():
+    L, d, b = 130, 8, 16
+    q, k, v = _rand(13, L, d)
+    nk = -(-L // b)
+    base = orc.sol_attn_forward(q, k, v, b, b, 0.7)
+    forced = np.zeros(nk, dtype=bool)
+    forced[[1, nk - 1]] = True
+    r = orc.sol_attn_forward(q, k, v, b, b, 0.7, forced=forced)
+    assert np.array_equal(r.mask, base.mask | forced[None, :])
+    np.testing.assert_allclose(r.out, orc.sol_attn_definition(q, k, v, r.mask, b, b), rtol=1e-11, atol=1e-12)
+    # forcing everything is dense attention whatever beta is
+    rall = orc.sol_attn_forward(q, k, v, b, b, math.inf, forced=np.ones(nk, dtype=bool))
+    ref = scipy_softmax((q @ k.T) / math.sqrt(d), axis=1) @ v
+    np.testing.assert_allclose(rall.out, ref, rtol=1e-11, atol=1e-12)
+    # the diagonal estimator changes sigma (hence tau) but not mu
+    rd = orc.routing(q, k, v, b, b, 0.7, estimator="diagonal")
+    np.testing.assert_allclose(rd.mu, base.mu, rtol=1e-12, atol=1e-14)
+    v_k = np.var(base.kc, axis=0)                                   # numpy's own per-channel variance
+    np.testing.assert_allclose(rd.sigma, np.sqrt((base.qbar ** 2) @ v_k) / math.sqrt(d), rtol=1e-10)
