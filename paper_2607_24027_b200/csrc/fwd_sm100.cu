@@ -44,23 +44,31 @@ constexpr int kHalf = 64;                        // key columns per softmax warp
 constexpr int kThreads = 384;
 constexpr int kTileBytes = kBlk * kD * 2;        // 32 KB: one K-like or V-like tile
 constexpr int kHalfBytes = kTileBytes / 2;       // 16 KB: 64 channels x 128 rows (one TMA box)
-constexpr int kStages = 4;                       // ring of K/V tiles
+constexpr int kKStages = 2;                      // ring of K tiles
+constexpr int kVStages = 2;                      // ring of V tiles (its own ring: the score GEMMs run ahead of P V)
+constexpr int kStages = kKStages + kVStages;
 constexpr int kGroup = 32;                       // pooled keys scored per router step (one per lane)
 constexpr int kRecords = 4;                      // ring of routing records
 constexpr int kTmemCols = 512;
 constexpr int kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units
-constexpr int kStaggerCycles = 0;                // head start of softmax group 0 over group 1, per work item
 
-constexpr uint8_t kRecFirst = 1, kRecLast = 2, kRecApprox = 4;
+// The router turns every chunk of 128 key blocks into a record: a flat list of tile descriptors
+// that the other roles only have to read.  A descriptor is (row coordinate << 5) | flags; the
+// coordinate is the first key row of an exact tile or the first pooled row of an approximate one.
+constexpr uint32_t kTileApprox = 1;      // approximate-branch tile (pooled keys / mean values)
+constexpr uint32_t kTileFirst = 2;       // first tile of its work item: Q_i is loaded, accumulators start afresh
+constexpr uint32_t kTileEnd = 4;         // not a tile: the work item ends here
+constexpr uint32_t kTileEmptyItem = 8;   // on an end entry: the item had no tile at all
+constexpr uint32_t kDescStop = 0xffffffffu, kDescAbort = 0xfffffffeu, kDescNone = 0xfffffffdu;
 
 struct alignas(16) Record {
   float bias[kBlk];             // approximate-tile column bias: log2(n_j) / (scale * log2 e), or -inf
   int32_t work;                 // bh * Nq + i, or -1: no more work
-  int16_t chunk;
-  uint8_t flags;
-  uint8_t n_sel;
-  uint8_t sel[kBlk];            // offsets (within the chunk) of the routed blocks
+  int32_t bh;
+  int32_t q_row;                // first query row of the work item
+  int16_t first, end;           // descriptors [first, end) are valid (slot 0 is kept for the approximate tile)
+  uint32_t desc[kBlk + 2];
 };
 
 struct Shared {
@@ -69,7 +77,7 @@ struct Shared {
   Record rec[kRecords];
   float2 ml[2][kBlk];           // (m_h, l_h) exchange between the softmax warpgroups
   uint64_t rec_full[kRecords], rec_empty[kRecords];
-  uint64_t kv_full[kStages], kv_empty[kStages];
+  uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
   uint64_t q_full, q_empty;
   uint64_t s_full[2], p_full[2][2], pv_done[2];   // indexed by score buffer (and warpgroup)
   uint64_t x_full, x_done;      // rendezvous of the two softmax warpgroups at the end of a work item
@@ -128,7 +136,7 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_FLUSH(role) prof.flush(role)
 #define PROF_ACC(slot) (&prof.v[slot])
 // timeline of a few tiles of CTA 0: [tile][event] = clock64()
-constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 12;
+constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 16;
 __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
 #define PROF_T0 const long long prof_t0 = clock64();
@@ -145,81 +153,41 @@ __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #endif
 
 // ------------------------------------------------------------------------------------------------
-// Walks the record ring and turns it into a flat stream of events: one per tile, one at the end of
-// every work item, one at the end of the stream.  The producer, the MMA thread and both softmax
-// warpgroups each run their own cursor over the same records.
-enum : int { kEvTile = 0, kEvItemEnd = 1, kEvEnd = 2, kEvAbort = 3 };
-struct Event {
-  int type;
-  int work;          // bh * Nq + i
-  int block;         // tile: key block index j (exact) or first block of the chunk (approximate)
-  bool approx;       // tile: approximate-branch tile
-  bool first;        // tile: first tile of its work item; item end: the item had no tile at all
-  const Record* rec; // tile: its record (bias of an approximate tile)
-};
-
+// Every consumer role (producer, the two MMA threads, both softmax warpgroups) walks the record
+// ring with a cursor of its own and sees the same flat stream of descriptors.
 struct Cursor {
   uint32_t n_rec = 0;
-  int e = 0;                 // next tile of the current record
-  int n_tiles = 0;
-  int work = 0;              // fields of the open record, cached in registers
-  int block0 = 0;
-  bool has_approx = false;
-  bool have = false;         // a record is open
-  bool item_has_tiles = false;
-  bool end_pending = false;
-  const Record* rec = nullptr;
+  int e = 0, end = 0;
+  const Record* rec = nullptr;   // the open record (valid until the next call)
 };
 
 // `release` is called when the cursor is done with a record (arrives on rec_empty as appropriate
-// for the role).  Returns kEvAbort when a bounded wait expired.
+// for the role).  Returns kDescStop at the end of the stream, kDescAbort when a bounded wait
+// expired and, with block = false, kDescNone when the next record has not been written yet.
 template <class Release>
-__device__ __forceinline__ Event next_event(Shared& sm, Cursor& c, long long* wait_acc, Release release) {
-  Event ev{};
+__device__ __forceinline__ uint32_t next_desc(Shared& sm, Cursor& c, long long* wait_acc, Release release,
+                                              bool block = true) {
   for (;;) {
-    if (!c.have) {
-      const uint32_t r = c.n_rec % kRecords;
+    if (c.e < c.end) return c.rec->desc[c.e++];
+    if (c.rec) {
+      release(c.n_rec % kRecords);
+      c.rec = nullptr;
+      ++c.n_rec;
+    }
+    const uint32_t r = c.n_rec % kRecords;
+    if (!block && !mbar_try_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1)) return kDescNone;
 #ifdef SOL_PROFILE
-      const long long t = clock64();
+    const long long t = clock64();
 #endif
-      const bool ok = mbar_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1, &sm.abort_flag);
+    const bool ok = mbar_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1, &sm.abort_flag);
 #ifdef SOL_PROFILE
-      if (wait_acc) *wait_acc += clock64() - t;
+    if (wait_acc) *wait_acc += clock64() - t;
 #endif
-      if (!ok) { ev.type = kEvAbort; return ev; }
-      c.rec = &sm.rec[r];
-      c.work = c.rec->work;
-      if (c.work < 0) { ev.type = kEvEnd; return ev; }
-      const uint32_t flags = c.rec->flags;
-      c.have = true;
-      c.e = 0;
-      c.has_approx = (flags & kRecApprox) != 0;
-      c.n_tiles = (c.has_approx ? 1 : 0) + c.rec->n_sel;
-      c.block0 = c.rec->chunk * kBlk;
-      if (flags & kRecFirst) c.item_has_tiles = false;
-      c.end_pending = (flags & kRecLast) != 0;
-    }
-    if (c.e < c.n_tiles) {
-      ev.type = kEvTile;
-      ev.work = c.work;
-      ev.approx = c.has_approx && c.e == 0;
-      ev.block = c.block0 + (ev.approx ? 0 : c.rec->sel[c.e - (c.has_approx ? 1 : 0)]);
-      ev.first = !c.item_has_tiles;
-      ev.rec = c.rec;
-      c.item_has_tiles = true;
-      ++c.e;
-      return ev;
-    }
-    if (c.end_pending) {
-      c.end_pending = false;
-      ev.type = kEvItemEnd;
-      ev.work = c.work;
-      ev.first = !c.item_has_tiles;
-      return ev;
-    }
-    release(c.n_rec % kRecords);
-    c.have = false;
-    ++c.n_rec;
+    if (!ok) return kDescAbort;
+    if (sm.rec[r].work < 0) return kDescStop;        // stays on this record: every further call stops too
+    c.rec = &sm.rec[r];
+    c.e = c.rec->first;
+    c.end = c.rec->end;
   }
 }
 
@@ -250,6 +218,7 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
     }
     const float* kc_head = p.kc + (size_t)bh * p.Nk * kD;
     int count = 0;
+    bool item_has_tiles = false;
     // Bulk-copy one group of 32 pooled keys (16 KB, contiguous in memory) into a staging buffer;
     // the copy of group n+1 is in flight while group n is scored.
     auto stage_group = [&](int jb) {
@@ -318,19 +287,27 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
         const bool valid = j < p.Nk;
         any_unselected |= (valid && !sel);
         rec.bias[g * 32 + lane] = (valid && !sel) ? log2f((float)min(kBlk, p.N - j * kBlk)) * inv_sl2 : -INFINITY;
-        if (sel) rec.sel[n_sel + __popc(m & ((1u << lane) - 1u))] = (uint8_t)(g * 32 + lane);
+        if (sel) rec.desc[1 + n_sel + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(j * kBlk) << 5;
         n_sel += __popc(m);
         if (p.mask_out && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
       }
       any_unselected = __any_sync(full, any_unselected);
       count += n_sel;
+      const bool has_approx = p.mode == SOL_MODE_SOL && any_unselected;
+      const int first = has_approx ? 0 : 1;
+      int end = 1 + n_sel;                   // n_sel <= 128
+      __syncwarp();
       if (lane == 0) {
         rec.work = w;
-        rec.chunk = (int16_t)t;
-        rec.n_sel = (uint8_t)n_sel;     // n_sel <= 128 fits
-        rec.flags = (t == 0 ? kRecFirst : 0) | (t == n_chunks - 1 ? kRecLast : 0) |
-                    ((p.mode == SOL_MODE_SOL && any_unselected) ? kRecApprox : 0);
+        rec.bh = bh;
+        rec.q_row = i * kBlk;
+        if (has_approx) rec.desc[0] = ((uint32_t)j0 << 5) | kTileApprox;
+        if (!item_has_tiles && end > first) rec.desc[first] |= kTileFirst;
+        if (t == n_chunks - 1) rec.desc[end] = kTileEnd | ((item_has_tiles || end > first) ? 0u : kTileEmptyItem);
+        rec.first = (int16_t)first;
+        rec.end = (int16_t)(end + (t == n_chunks - 1 ? 1 : 0));
       }
+      item_has_tiles |= end > first;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.rec_full[n_rec % kRecords]);
       ++n_rec;
@@ -352,52 +329,106 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// producer: one thread
+// producer: one thread.  K and V tiles have rings of their own, and the K loads run kLead tiles
+// ahead of the V loads: that is the order in which the slots come free (a K slot when its score
+// GEMM retires, a V slot a softmax pass and a P V later), so an in-order thread seldom waits for a
+// slot while another load could go.
 __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV,
                               const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vm) {
-  uint32_t n_load = 0, n_item = 0;
-  Cursor cur;
+  constexpr int kLead = 2;
+  uint32_t n_k = 0, n_v = 0, n_item = 0;
+  Cursor cur_k, cur_v;
   PROF_DECL
-  auto load_tile = [&](const CUtensorMap* tm, int row, int bh) -> bool {
-    const uint32_t s = n_load % kStages;
-    if (!WAIT(&sm.kv_empty[s], ((n_load / kStages) & 1) ^ 1, 1)) return false;   // prof 1: K/V ring full
-    mbar_arrive_expect_tx(&sm.kv_full[s], kTileBytes);
-    unsigned char* dst = sKV + (size_t)s * kTileBytes;
-    tma_load_3d(dst, tm, &sm.kv_full[s], 0, row, bh);
-    tma_load_3d(dst + kHalfBytes, tm, &sm.kv_full[s], 64, row, bh);
-    ++n_load;
-    return true;
+  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, int bh) {
+    mbar_arrive_expect_tx(full, kTileBytes);
+    tma_load_3d(dst, tm, full, 0, row, bh);
+    tma_load_3d(dst + kHalfBytes, tm, full, 64, row, bh);
   };
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
-  int item_loaded = -1;
+  bool k_end = false, have_k = false, ok = true;
+  uint32_t dk = 0;
   for (;;) {
-    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                 // prof 0: no record yet
-    if (ev.type == kEvEnd) break;
-    if (ev.type == kEvAbort) { flag_abort(sm, p, 200); break; }
-    const int bh = ev.work / p.Nq, i = ev.work - bh * p.Nq;
-    if (ev.work != item_loaded) {
-      // Q_i for this work item (also for an item without tiles, to keep the phases in step)
-      if (!WAIT(&sm.q_empty, (n_item & 1) ^ 1, 2)) { flag_abort(sm, p, 201); break; }   // prof 2: Q slot busy
-      mbar_arrive_expect_tx(&sm.q_full, kTileBytes);
-      tma_load_3d(sQ, tm_q, &sm.q_full, 0, i * kBlk, bh);
-      tma_load_3d(sQ + kHalfBytes, tm_q, &sm.q_full, 64, i * kBlk, bh);
-      ++n_item;
-      item_loaded = ev.work;
+    // K side (and Q): up to kLead tiles ahead of the V side
+    while (!k_end && (int)(n_k - n_v) < kLead) {
+      if (!have_k) {
+        // never sleep on the router while a V load is owed: the router may itself be waiting for
+        // the V cursor to hand a record back
+        dk = next_desc(sm, cur_k, PROF_ACC(0), release, n_k == n_v);            // prof 0: no record yet
+        if (dk == kDescNone) break;
+        if (dk == kDescAbort) { ok = false; break; }
+        if (dk == kDescStop) { k_end = true; break; }
+        have_k = true;
+      }
+      if (dk & kTileEnd) { have_k = false; continue; }
+      const int bh = cur_k.rec->bh;
+      if (dk & kTileFirst) {
+        // Q_i for this work item.  The slot frees when the previous item's last score GEMM
+        // retires; until then serve the V side.
+        const uint32_t par = (n_item & 1) ^ 1;
+        if (n_k != n_v && !mbar_try_wait(&sm.q_empty, par)) break;
+        if (!WAIT(&sm.q_empty, par, 2)) { ok = false; break; }                  // prof 2: Q slot busy
+        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, bh);
+        ++n_item;
+        dk &= ~kTileFirst;
+      }
+      have_k = false;
+      const uint32_t s = n_k % kKStages;
+      if (!WAIT(&sm.k_empty[s], ((n_k / kKStages) & 1) ^ 1, 1)) { ok = false; break; }   // prof 1: K ring full
+      {
+        PROF_T0
+        load_tile((dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes, (int)(dk >> 5), bh);
+        PROF_ADD(4)                                                                    // prof 4: issuing K copies
+      }
+      TRACE(n_k, 12);
+      ++n_k;
     }
-    if (ev.type != kEvTile) continue;
-    bool ok;
-    if (ev.approx) ok = load_tile(tm_kc, ev.block, bh) && load_tile(tm_vm, ev.block, bh);
-    else ok = load_tile(tm_k, ev.block * kBlk, bh) && load_tile(tm_v, ev.block * kBlk, bh);
-    if (!ok) { flag_abort(sm, p, 202); break; }
+    if (!ok) break;
+    if (n_k == n_v) {
+      if (k_end) break;
+      continue;
+    }
+    // V side: the oldest tile whose K is already on its way
+    uint32_t dv;
+    {
+      PROF_T0
+      do {
+        dv = next_desc(sm, cur_v, nullptr, release);
+      } while (dv < kDescNone && (dv & kTileEnd));
+      PROF_ADD(6)                                                                      // prof 6: V cursor
+    }
+    if (dv >= kDescNone) { ok = false; break; }          // cannot end before the K side did
+    const uint32_t s = n_v % kVStages;
+    if (!WAIT(&sm.v_empty[s], ((n_v / kVStages) & 1) ^ 1, 3)) { ok = false; break; }     // prof 3: V ring full
+    {
+      PROF_T0
+      load_tile((dv & kTileApprox) ? tm_vm : tm_v, &sm.v_full[s], sKV + (size_t)(kKStages + s) * kTileBytes,
+                (int)(dv >> 5), cur_v.rec->bh);
+      PROF_ADD(5)                                                                      // prof 5: issuing V copies
+    }
+    TRACE(n_v, 13);
+    ++n_v;
+  }
+  if (ok) {
+    // the V cursor still has to hand back the records that hold no further tile
+    for (;;) {
+      const uint32_t dv = next_desc(sm, cur_v, nullptr, release);
+      if (dv >= kDescNone) break;
+    }
+  } else {
+    flag_abort(sm, p, 200);
   }
   PROF_FLUSH(1);
   if (sm.abort_flag) {
     // let copies that are still in flight land before the CTA's shared memory goes away
     int never = 0;                                   // this drain must not be cut short by the abort flag
-    for (uint32_t back = 0; back < kStages && back < n_load; ++back) {
-      const uint32_t n = n_load - 1 - back;
-      mbar_wait(&sm.kv_full[n % kStages], (n / kStages) & 1, &never);
+    for (uint32_t back = 0; back < kKStages && back < n_k; ++back) {
+      const uint32_t n = n_k - 1 - back;
+      mbar_wait(&sm.k_full[n % kKStages], (n / kKStages) & 1, &never);
+    }
+    for (uint32_t back = 0; back < kVStages && back < n_v; ++back) {
+      const uint32_t n = n_v - 1 - back;
+      mbar_wait(&sm.v_full[n % kVStages], (n / kVStages) & 1, &never);
     }
   }
 }
@@ -420,29 +451,30 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
   const uint32_t q_lo = (smem_addr(sQ) >> 4) | (1u << 16);
   const uint32_t kv_lo = (smem_addr(sKV) >> 4) | (1u << 16);
   uint32_t n_item = 0, g = 0;
-  uint32_t slot = 0, slot_parity = 0;          // ring position of K(g): load 2g
+  uint32_t slot = 0, slot_parity = 0;          // ring position of K(g)
   Cursor cur;
   PROF_DECL
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
-  int item_seen = -1;
   for (;;) {
-    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                       // prof 0: no record yet
-    if (ev.type == kEvAbort) { ok = false; break; }
-    if (ev.type == kEvEnd) break;
-    if (ev.work != item_seen) {
-      if (!WAIT(&sm.q_full, n_item & 1, 1)) { ok = false; break; }                    // prof 1: Q not loaded
-      ++n_item;
-      item_seen = ev.work;
-    }
-    if (ev.type == kEvItemEnd) {                  // every MMA that reads Q_i has been issued
-      mma_commit(&sm.q_empty);
+    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
+    if (dsc == kDescAbort) { ok = false; break; }
+    if (dsc == kDescStop) break;
+    if (dsc & kTileEnd) {                         // every MMA that reads Q_i has been issued
+      if (!(dsc & kTileEmptyItem)) mma_commit(&sm.q_empty);
       continue;
     }
+    if (dsc & kTileFirst) {
+      if (!WAIT(&sm.q_full, n_item & 1, 1)) { ok = false; break; }                    // prof 1: Q not loaded
+      ++n_item;
+    }
     const uint32_t b = g & 1;
-    if (!WAIT(&sm.kv_full[slot], slot_parity, 2)) { ok = false; break; }              // prof 2: K not loaded
-    // the previous user of this score buffer was tile g-2: its P V must have read P out of it
-    if (g >= 2 && !WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }   // prof 3: score buffer busy
+    if (!WAIT(&sm.k_full[slot], slot_parity, 2)) { ok = false; break; }               // prof 2: K not loaded
+    TRACE(g, 14);
+    if (g >= 2) {
+      // P overwrites S: the P V of tile g-2 must have read P out of this buffer
+      if (!WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }        // prof 3: score buffer busy
+    }
     tc_fence_after();
     TRACE(g, 0);
     {
@@ -454,38 +486,38 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
         const uint32_t off = ((ks / 4) * kHalfBytes + (ks % 4) * 32) >> 4;
         mma_ss(d_tmem, desc_from_lo(q_lo + off), desc_from_lo(k_lo + off), idesc_qk, ks > 0);
       }
-      mma_commit(&sm.kv_empty[slot]);
+      mma_commit(&sm.k_empty[slot]);
       mma_commit(&sm.s_full[b]);
       PROF_ADD(6)                                                                      // prof 6: issuing Q K^T
     }
     TRACE(g, 1);
     ++g;
-    slot += 2;                                    // K tiles sit at every other ring position
-    if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
+    if (++slot == kKStages) { slot = 0; slot_parity ^= 1; }
   }
   if (!ok) flag_abort(sm, p, 300);
   PROF_FLUSH(2);
 }
 
-// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11, one thread)
+// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11, one thread); the fixed-reference variant has
+// one accumulator and P in its own columns
 __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uint32_t tmem) {
   const uint32_t idesc_pv = make_idesc_bf16(kBlk, kD, false, true);
-  const uint32_t kv_lo = (smem_addr(sKV) >> 4) | ((uint32_t)(kHalfBytes >> 4) << 16);
+  const uint32_t kv_lo = (smem_addr(sKV + kKStages * kTileBytes) >> 4) | ((uint32_t)(kHalfBytes >> 4) << 16);
   uint32_t g = 0;
-  uint32_t slot = 1, slot_parity = 0;          // ring position of V(g): load 2g+1
+  uint32_t slot = 0, slot_parity = 0;          // ring position of V(g)
   Cursor cur;
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const Event ev = next_event(sm, cur, nullptr, release);
-    if (ev.type == kEvAbort) { ok = false; break; }
-    if (ev.type == kEvEnd) break;
-    if (ev.type != kEvTile) continue;
+    const uint32_t dsc = next_desc(sm, cur, nullptr, release);
+    if (dsc == kDescAbort) { ok = false; break; }
+    if (dsc == kDescStop) break;
+    if (dsc & kTileEnd) continue;
     const uint32_t b = g & 1;
-    if (!mbar_wait(&sm.kv_full[slot], slot_parity, &sm.abort_flag)) { ok = false; break; }
+    if (!mbar_wait(&sm.v_full[slot], slot_parity, &sm.abort_flag)) { ok = false; break; }
     TRACE(g, 2);
     const uint32_t v_lo = kv_lo + slot * (kTileBytes >> 4);
-    const uint32_t acc_first = ev.first ? 0u : 1u;
+    const uint32_t acc_first = (dsc & kTileFirst) ? 0u : 1u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag)) { ok = false; break; }
@@ -493,24 +525,25 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < kHalf / 16; ++ks) {
-        mma_ts(tmem + kTmemO + h * kD, tmem + kTmemS + b * kBlk + h * kHalf + ks * 8,
-               desc_from_lo(v_lo + ((h * (kHalf * 128) + ks * 2048) >> 4)), idesc_pv, ks > 0 ? 1u : acc_first);
+        const uint32_t d_o = tmem + kTmemO + h * kD;
+        const uint32_t a_p = tmem + kTmemS + b * kBlk + h * kHalf + ks * 8;
+        const uint32_t acc = ks > 0 ? 1u : acc_first;
+        mma_ts(d_o, a_p, desc_from_lo(v_lo + ((h * (kHalf * 128) + ks * 2048) >> 4)), idesc_pv, acc);
       }
     }
     if (!ok) break;
-    mma_commit(&sm.kv_empty[slot]);
+    mma_commit(&sm.v_empty[slot]);
     mma_commit(&sm.pv_done[b]);
     TRACE(g, 5);
     ++g;
-    slot += 2;
-    if (slot >= kStages) { slot -= kStages; slot_parity ^= 1; }
+    if (++slot == kVStages) { slot = 0; slot_parity ^= 1; }
   }
   if (!ok) flag_abort(sm, p, 301);
 }
 
 // ------------------------------------------------------------------------------------------------
 // softmax + correction + epilogue: two warpgroups of 128 threads; thread = query row, warpgroup h
-// owns key columns [64h, 64h+64) of every tile
+// owns key columns [64h, 64h+64) of every tile.
 __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, int warp_in_group, int lane) {
   const unsigned full = 0xffffffffu;
   const uint32_t lane_base = tmem + ((uint32_t)(warp_in_group * 32) << 16);
@@ -519,7 +552,6 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
   const int row = warp_in_group * 32 + lane;
   const float sl2 = p.scale * 1.4426950408889634f;
   uint32_t g = 0, n_merge = 0;
-  bool stagger = true;
   float m_used = -INFINITY, l = 0.f;
   Cursor cur;
   PROF_DECL
@@ -528,25 +560,16 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     if (lane == 0) mbar_arrive(&sm.rec_empty[r]);
   };
   for (;;) {
-    const Event ev = next_event(sm, cur, PROF_ACC(0), release);                       // prof 0: no record yet
-    if (ev.type == kEvEnd) break;
-    if (ev.type == kEvAbort) { flag_abort(sm, p, 400); break; }
+    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
+    if (dsc == kDescStop) break;
+    if (dsc == kDescAbort) { flag_abort(sm, p, 400); break; }
+    const bool first = (dsc & kTileFirst) != 0;
 
-    if (ev.type == kEvTile) {
-      if (stagger) {
-        // The two groups leave the end-of-item rendezvous in lockstep and would then hit the MUFU
-        // unit in the same phase of every tile; holding group 1 back by about half a tile keeps
-        // one group's exponentials under the other's loads, maxima and stores.
-        stagger = false;
-        if (h == 1 && kStaggerCycles > 0) {
-          const long long t_start = clock64();
-          while (clock64() - t_start < kStaggerCycles) {}
-        }
-      }
+    if (!(dsc & kTileEnd)) {
       const uint32_t b = g & 1;
       const uint32_t t_s = lane_base + kTmemS + b * kBlk + h * kHalf;
-      const bool approx = ev.approx;
-      const int cols_valid = approx ? kBlk : min(kBlk, p.N - ev.block * kBlk);
+      const bool approx = (dsc & kTileApprox) != 0;
+      const int cols_valid = approx ? kBlk : min(kBlk, p.N - (int)(dsc >> 5));
       const bool general = approx || cols_valid < kBlk;
       if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
       tc_fence_after();
@@ -562,7 +585,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         // bring the rare tiles (approximate chunk, ragged last block) to the common form
         // logit = sl2 * x by folding the column bias into x; -inf marks masked columns
         if (approx) {
-          const float4* bias4 = reinterpret_cast<const float4*>(&ev.rec->bias[h * kHalf]);
+          const float4* bias4 = reinterpret_cast<const float4*>(&cur.rec->bias[h * kHalf]);
 #pragma unroll
           for (int c = 0; c < kHalf / 4; ++c) {
             const float4 bb = bias4[c];
@@ -590,7 +613,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sl2;       // -inf when the whole half is masked
       }
       // ---- running maximum, lazy rescale of O_h
-      if (ev.first) {
+      if (first) {
         m_used = mx;
         l = 0.f;
       } else if (__any_sync(full, mx > m_used + kRescaleThreshold)) {
@@ -650,11 +673,11 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     }
 
     // ---- end of the work item: merge the two partial results, O_i = (w0 O0 + w1 O1) / (w0 l0 + w1 l1)
-    const int bh = ev.work / p.Nq, i = ev.work - bh * p.Nq;
-    const int q_rows = min(kBlk, p.N - i * kBlk);
-    __nv_bfloat16* orow = p.out + ((size_t)bh * p.N + (size_t)i * kBlk + row) * kD + h * kHalf;
+    const int q_row = cur.rec->q_row;
+    const int q_rows = min(kBlk, p.N - q_row);
+    __nv_bfloat16* orow = p.out + ((size_t)cur.rec->bh * p.N + (size_t)(q_row + row)) * kD + h * kHalf;
     PROF_T0
-    if (!ev.first) {
+    if (!(dsc & kTileEmptyItem)) {
       // the last P V of the item (one commit covers both halves)
       if (!WAIT(&sm.pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, 3)) { flag_abort(sm, p, 403); break; }   // prof 3
       tc_fence_after();
@@ -700,7 +723,6 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       mbar_arrive(&sm.x_done);
       if (!WAIT(&sm.x_done, n_merge & 1, 6)) { flag_abort(sm, p, 405); break; }
       ++n_merge;
-      stagger = true;
     } else if (row < q_rows) {
       // a query block that routed nothing in keep-or-drop mode has no attention mass at all
       for (int c = 0; c < kHalf; c += 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
@@ -725,9 +747,10 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     sm.abort_flag = 0;
-    // a record is released by the producer, the two MMA threads and the 8 softmax warps
-    for (int r = 0; r < kRecords; ++r) { mbar_init(&sm.rec_full[r], 1); mbar_init(&sm.rec_empty[r], 11); }
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
+    // a record is released by the two producers, the two MMA threads and the 8 softmax warps
+    for (int r = 0; r < kRecords; ++r) { mbar_init(&sm.rec_full[r], 1); mbar_init(&sm.rec_empty[r], 12); }
+    for (int s = 0; s < kKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kVStages; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
     mbar_init(&sm.q_full, 1); mbar_init(&sm.q_empty, 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm.s_full[b], 1);
@@ -785,7 +808,8 @@ bool fwd_sm100_supports(const Problem& p) { return p.d == kD && p.block_q == kBl
 
 cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, __nv_bfloat16* out, const WsPtrs& ws, const float* tau,
-                             int32_t* counts, uint32_t* mask_out, cudaStream_t stream, int* n_launches) {
+                             int32_t* counts, uint32_t* mask_out, cudaStream_t stream,
+                             int* n_launches) {
   CUtensorMap tq, tk, tv, tkc, tvm;
   if (!make_tmap_bf16_3d(&tq, q, p.BH, p.N, kD, kBlk) || !make_tmap_bf16_3d(&tk, k, p.BH, p.N, kD, kBlk) ||
       !make_tmap_bf16_3d(&tv, v, p.BH, p.N, kD, kBlk) || !make_tmap_bf16_3d(&tkc, ws.kcb, p.BH, p.Nk, kD, kBlk) ||
