@@ -49,6 +49,7 @@ constexpr int kVStages = 2;                      // ring of V tiles (its own rin
 constexpr int kStages = kKStages + kVStages;
 constexpr int kGroup = 32;                       // pooled keys scored per router step (one per lane)
 constexpr int kRecords = 4;                      // ring of routing records
+constexpr int kWarpRouter = 8, kWarpProducer = 9, kWarpQK = 10;   // warp 11 issues P V
 constexpr int kTmemCols = 512;
 constexpr int kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units
@@ -136,7 +137,7 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_FLUSH(role) prof.flush(role)
 #define PROF_ACC(slot) (&prof.v[slot])
 // timeline of a few tiles of CTA 0: [tile][event] = clock64()
-constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 16;
+constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 32;
 __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
 #define PROF_T0 const long long prof_t0 = clock64();
@@ -469,12 +470,14 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
       ++n_item;
     }
     const uint32_t b = g & 1;
+    TRACE(g, 24);
     if (!WAIT(&sm.k_full[slot], slot_parity, 2)) { ok = false; break; }               // prof 2: K not loaded
     TRACE(g, 14);
     if (g >= 2) {
       // P overwrites S: the P V of tile g-2 must have read P out of this buffer
       if (!WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }        // prof 3: score buffer busy
     }
+    TRACE(g, 25);
     tc_fence_after();
     TRACE(g, 0);
     {
@@ -639,22 +642,25 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       //      TMEM over the start of the half
       {
         const float nm = (m_used == -INFINITY) ? 0.f : -m_used;   // a half that has seen nothing yet: all P = 0
-        const uint64_t sl2_2 = pack2(sl2, sl2), nm2 = pack2(nm, nm);
-        uint64_t s_a = pack2(0.f, 0.f), s_b = pack2(0.f, 0.f);
+        const float2 sl2_2 = make_float2(sl2, sl2), nm2 = make_float2(nm, nm);
+        float2 s_a = make_float2(0.f, 0.f), s_b = make_float2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < kHalf; c += 4) {
-          float xa, xb, xc, xd;
-          unpack2(fma2(pack2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sl2_2, nm2), xa, xb);
-          unpack2(fma2(pack2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sl2_2, nm2), xc, xd);
-          const float e0 = ex2(xa), e1 = ex2(xb), e2 = ex2(xc), e3 = ex2(xd);
-          s_a = add2(s_a, pack2(e0, e1));
-          s_b = add2(s_b, pack2(e2, e3));
-          __nv_bfloat162 lo = __floats2bfloat162_rn(e0, e1);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(e2, e3);
+          const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sl2_2, nm2);
+          const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sl2_2, nm2);
+          const float2 ea = make_float2(ex2(xa.x), ex2(xa.y));
+          const float2 eb = make_float2(ex2(xb.x), ex2(xb.y));
+          s_a = __fadd2_rn(s_a, ea);
+          s_b = __fadd2_rn(s_b, eb);
+          __nv_bfloat162 lo = __floats2bfloat162_rn(ea.x, ea.y);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(eb.x, eb.y);
           sr[c / 2] = *reinterpret_cast<uint32_t*>(&lo);
           sr[c / 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
         }
-        { float t0, t1; unpack2(add2(s_a, s_b), t0, t1); l += t0 + t1; }
+        {
+          const float2 t = __fadd2_rn(s_a, s_b);
+          l += t.x + t.y;
+        }
         tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
       }
       PROF_ADD(8)                                                                      // prof 8: load + arithmetic
@@ -663,6 +669,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       tc_fence_before();
       mbar_arrive(&sm.p_full[h][b]);
       if (row == 0) TRACE(g, 8 + 3 * h);
+      if (lane == 0) TRACE(g, 16 + 4 * h + warp_in_group);
       PROF_ADD(9)                                                                      // prof 9: whole tile
 #ifdef SOL_PROFILE
       if (approx) { prof.v[10] += clock64() - prof_t0; ++prof.v[0]; }                  // prof 10 / 0: approximate tiles: cycles / count
@@ -762,7 +769,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     mbar_init(&sm.kc_full[0], 1); mbar_init(&sm.kc_full[1], 1);
     fence_mbar_init();
   }
-  if (warp == 9 && lane == 0) {
+  if (warp == kWarpProducer && lane == 0) {
     prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
     prefetch_tensormap(&tm_kc); prefetch_tensormap(&tm_vm);
   }
@@ -774,11 +781,11 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (warp < 8) {
     softmax_role(sm, p, tmem, warp / 4, warp % 4, lane);
-  } else if (warp == 8) {
+  } else if (warp == kWarpRouter) {
     router_role(sm, p, lane);
-  } else if (warp == 9) {
+  } else if (warp == kWarpProducer) {
     if (lane == 0) producer_role(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
-  } else if (warp == 10) {
+  } else if (warp == kWarpQK) {
     if (lane == 0) mma_qk_role(sm, p, sQ, sKV, tmem);
   } else {
     if (lane == 0) mma_pv_role(sm, p, sKV, tmem);
