@@ -72,6 +72,14 @@ enum {
   SOL_IMPL_MMA_SYNC = 2   /* portable warp-level mma.sync kernel (all supported shapes)        */
 };
 
+/* memory layout of q, k, v and out (all four the same); d channels of a token are contiguous */
+enum {
+  SOL_LAYOUT_BHND = 0,    /* [B, H, N, d] row-major: the paper's per-head view (default)         */
+  SOL_LAYOUT_BNHD = 1     /* [B, N, H, d] row-major: what a fused QKV projection of a DiT block
+                             leaves behind; the heads of a token are interleaved, no transpose
+                             is needed before or after the operator                              */
+};
+
 /* Human-readable name of a status code; never NULL, static storage. */
 const char* sol_attn_status_string(sol_status_t status);
 
@@ -146,6 +154,7 @@ typedef struct {
                                                    (text / sink key-value tokens kept exact, as in
                                                    the paper's MMDiT integrations); shared by all
                                                    batches and heads; counts include them         */
+  int32_t layout;                               /* SOL_LAYOUT_* of q, k, v and out (0 = [B,H,N,d]) */
 } sol_attn_args;
 sol_status_t sol_attn_forward_ex(const sol_attn_args* args /* host */);
 

@@ -38,7 +38,8 @@ sol_status_t check_shape(int B, int H, int N, int d, int block_q, int block_k, b
 }
 
 sol::Problem make_problem(int B, int H, int N, int d, int block_q, int block_k, float beta, float scale, int mode,
-                          int estimator = SOL_EST_MOMENTS, const uint8_t* forced = nullptr) {
+                          int estimator = SOL_EST_MOMENTS, const uint8_t* forced = nullptr,
+                          int layout = SOL_LAYOUT_BHND) {
   sol::Problem p{};
   p.B = B; p.H = H; p.N = N; p.d = d; p.block_q = block_q; p.block_k = block_k;
   p.BH = B * H;
@@ -49,6 +50,12 @@ sol::Problem make_problem(int B, int H, int N, int d, int block_q, int block_k, 
   p.mode = mode;
   p.estimator = estimator;
   p.forced = forced;
+  p.st.H = H;
+  if (layout == SOL_LAYOUT_BNHD) {
+    p.st.row = (long long)H * d; p.st.head = d; p.st.batch = (long long)N * H * d;
+  } else {
+    p.st.row = d; p.st.head = (long long)N * d; p.st.batch = (long long)H * N * d;
+  }
   return p;
 }
 
@@ -131,13 +138,14 @@ sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
   if (a->mode != SOL_MODE_DENSE && !a->tau_override && std::isnan(a->threshold)) return SOL_ERR_INVALID_ARG;
   if (std::isnan(a->scale) || std::isinf(a->scale)) return SOL_ERR_INVALID_ARG;
   if (a->estimator != SOL_EST_MOMENTS && a->estimator != SOL_EST_DIAGONAL) return SOL_ERR_INVALID_ARG;
+  if (a->layout != SOL_LAYOUT_BHND && a->layout != SOL_LAYOUT_BNHD) return SOL_ERR_INVALID_ARG;
   if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 1023u) != 0) return SOL_ERR_WORKSPACE;
   if (a->workspace_bytes < sol_attn_workspace_bytes(a->B, a->H, a->N, a->d, a->block_q, a->block_k))
     return SOL_ERR_WORKSPACE;
   if ((s = check_arch()) != SOL_OK) return s;
 
   const sol::Problem p = make_problem(a->B, a->H, a->N, a->d, a->block_q, a->block_k, a->threshold, a->scale, a->mode,
-                                      a->estimator, a->mode == SOL_MODE_DENSE ? nullptr : a->forced_blocks);
+                                      a->estimator, a->mode == SOL_MODE_DENSE ? nullptr : a->forced_blocks, a->layout);
   int impl = a->impl;
   if (impl == SOL_IMPL_AUTO) impl = sol::fwd_sm100_supports(p) ? SOL_IMPL_TCGEN05 : SOL_IMPL_MMA_SYNC;
   if (impl == SOL_IMPL_TCGEN05 && !sol::fwd_sm100_supports(p)) return SOL_ERR_UNSUPPORTED_SHAPE;

@@ -20,6 +20,17 @@ constexpr int kCovSlices = 4;         // partial second-moment matrices per (bat
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Where element (b, h, n, 0) of q, k, v and out sits (all four share one layout): element strides
+// between consecutive tokens, heads and batches.  A token's d channels are always contiguous.
+struct Strides {
+  long long row, head, batch;
+  int H;
+  __host__ __device__ size_t base(int bh) const {
+    const int b = bh / H;
+    return (size_t)b * (size_t)batch + (size_t)(bh - b * H) * (size_t)head;
+  }
+};
+
 // One attention problem and where its pre-attention results live.
 struct Problem {
   int B, H, N, d, block_q, block_k;
@@ -29,6 +40,7 @@ struct Problem {
   int mode;          // SOL_MODE_*
   int estimator;     // SOL_EST_*: how sigma_i is obtained
   const uint8_t* forced;   // device [Nk] or null: key blocks that always go to the exact branch
+  Strides st;              // SOL_LAYOUT_*: strides of q, k, v, out
 };
 
 // Byte offsets into the workspace (all multiples of 1024).

@@ -60,13 +60,15 @@ struct Smem {
   int any_unselected;
 };
 
-// Copy `rows` rows of D bf16 from global into a padded shared tile; rows beyond are zeroed.
+// Copy `rows` rows of D bf16 (row_stride elements apart) from global into a padded shared tile;
+// rows beyond are zeroed.
 template <int D, int BLK, int THREADS>
-__device__ __forceinline__ void load_tile(__nv_bfloat16 (*dst)[D + 8], const __nv_bfloat16* src, int rows) {
+__device__ __forceinline__ void load_tile(__nv_bfloat16 (*dst)[D + 8], const __nv_bfloat16* src, int rows,
+                                          size_t row_stride) {
   constexpr int CPR = D / 8;                    // 16-byte chunks per row
   for (int e = threadIdx.x; e < BLK * CPR; e += THREADS) {
     const int r = e / CPR, c = e % CPR;
-    if (r < rows) cp_async16(&dst[r][c * 8], src + (size_t)r * D + c * 8);
+    if (r < rows) cp_async16(&dst[r][c * 8], src + (size_t)r * row_stride + c * 8);
     else *reinterpret_cast<uint4*>(&dst[r][c * 8]) = make_uint4(0, 0, 0, 0);
   }
 }
@@ -76,8 +78,8 @@ __global__ void __launch_bounds__(BLK * 2)
 fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ out,
                     WsPtrs ws, const float* __restrict__ tau, int32_t* __restrict__ counts,
-                    uint32_t* __restrict__ mask_out, const uint8_t* __restrict__ forced, int N, int Nq, int Nk,
-                    float scale, int mode) {
+                    uint32_t* __restrict__ mask_out, const uint8_t* __restrict__ forced, Strides st, int N, int Nq,
+                    int Nk, float scale, int mode) {
   constexpr int THREADS = BLK * 2;
   constexpr int WARPS = THREADS / 32;
   constexpr int NT = BLK / 8;                   // score n-tiles (8 key columns each)
@@ -93,7 +95,8 @@ fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   const float scale_log2 = scale * 1.4426950408889634f;
 
   // ---- stage Q_i, build its A fragments (kept in registers for the whole kernel)
-  load_tile<D, BLK, THREADS>(sm.k, q + ((size_t)bh * N + q_row0) * D, q_rows);
+  const size_t head_base = st.base(bh);          // element offset of (b, h, token 0) in q, k, v, out
+  load_tile<D, BLK, THREADS>(sm.k, q + head_base + (size_t)q_row0 * st.row, q_rows, st.row);
   if (mode != SOL_MODE_DENSE)
     for (int c = threadIdx.x; c < D; c += THREADS) sm.qbar[c] = ws.qbar[((size_t)bh * Nq + i) * D + c];
   cp_async_wait_all();
@@ -120,9 +123,10 @@ fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   //   approx = true : columns are pooled keys, bias[col] = log2(n_j) or -inf (selected / padding)
   //   approx = false: columns are tokens, columns >= cols_valid are -inf
   auto process_tile = [&](const __nv_bfloat16* ksrc, const __nv_bfloat16* vsrc, int cols_valid, bool approx) {
+    const size_t rs = approx ? (size_t)D : (size_t)st.row;   // pooled operands are dense [Nk][D]
     __syncthreads();                            // everyone is done with the previous tile
-    load_tile<D, BLK, THREADS>(sm.k, ksrc, cols_valid);
-    load_tile<D, BLK, THREADS>(sm.v, vsrc, cols_valid);
+    load_tile<D, BLK, THREADS>(sm.k, ksrc, cols_valid, rs);
+    load_tile<D, BLK, THREADS>(sm.v, vsrc, cols_valid, rs);
     cp_async_wait_all();
     __syncthreads();
 
@@ -250,7 +254,7 @@ fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                    min(BLK, Nk - j0), true);
     for (int e = 0; e < n_sel; ++e) {                      // exact branch, inner loop
       const int j = j0 + sm.sel_list[e];
-      process_tile(k + ((size_t)bh * N + (size_t)j * BLK) * D, v + ((size_t)bh * N + (size_t)j * BLK) * D,
+      process_tile(k + head_base + (size_t)j * BLK * st.row, v + head_base + (size_t)j * BLK * st.row,
                    min(BLK, N - j * BLK), false);
     }
   }
@@ -264,14 +268,14 @@ fwd_mma_sync_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
   const float inv0 = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f;
   const float inv1 = l_run[1] > 0.f ? 1.f / l_run[1] : 0.f;
   const int r0 = warp * 16 + lane / 4, r1 = r0 + 8;
-  __nv_bfloat16* obase = out + ((size_t)bh * N + q_row0) * D;
+  __nv_bfloat16* obase = out + head_base + (size_t)q_row0 * st.row;
 #pragma unroll
   for (int dn = 0; dn < DN; ++dn) {
     const int c = dn * 8 + (lane % 4) * 2;
     if (r0 < q_rows)
-      *reinterpret_cast<uint32_t*>(obase + (size_t)r0 * D + c) = pack_bf16(o_acc[dn][0] * inv0, o_acc[dn][1] * inv0);
+      *reinterpret_cast<uint32_t*>(obase + (size_t)r0 * st.row + c) = pack_bf16(o_acc[dn][0] * inv0, o_acc[dn][1] * inv0);
     if (r1 < q_rows)
-      *reinterpret_cast<uint32_t*>(obase + (size_t)r1 * D + c) = pack_bf16(o_acc[dn][2] * inv1, o_acc[dn][3] * inv1);
+      *reinterpret_cast<uint32_t*>(obase + (size_t)r1 * st.row + c) = pack_bf16(o_acc[dn][2] * inv1, o_acc[dn][3] * inv1);
   }
   if (threadIdx.x == 0 && counts) counts[(size_t)bh * Nq + i] = count;
 }
@@ -286,7 +290,7 @@ cudaError_t launch_impl(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
   if (e != cudaSuccess) return e;
   dim3 grid(p.Nq, p.BH);
   fwd_mma_sync_kernel<D, BLK><<<grid, BLK * 2, smem, stream>>>(q, k, v, out, ws, tau, counts, mask_out, p.forced,
-                                                                p.N, p.Nq, p.Nk, p.scale, p.mode);
+                                                                p.st, p.N, p.Nq, p.Nk, p.scale, p.mode);
   return cudaGetLastError();
 }
 

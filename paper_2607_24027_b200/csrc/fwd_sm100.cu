@@ -66,7 +66,7 @@ constexpr uint32_t kDescStop = 0xffffffffu, kDescAbort = 0xfffffffeu, kDescNone 
 struct alignas(16) Record {
   float bias[kBlk];             // approximate-tile column bias: log2(n_j) / (scale * log2 e), or -inf
   int32_t work;                 // bh * Nq + i, or -1: no more work
-  int32_t bh;
+  int32_t b, h;                 // batch and head of the work item
   int32_t q_row;                // first query row of the work item
   int16_t first, end;           // descriptors [first, end) are valid (slot 0 is kept for the approximate tile)
   uint32_t desc[kBlk + 2];
@@ -98,6 +98,8 @@ struct Params {
   int N, Nq, Nk, total_work, mode;
   float scale;
   const uint8_t* forced;        // [Nk] or null: key blocks always routed to the exact branch
+  Strides st;                   // layout of q, k, v, out
+  int rows_inner;               // coordinate order of the q/k/v tensor maps: (c, row, h, b) or (c, h, row, b)
 };
 
 __device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int where) {
@@ -300,7 +302,8 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
       __syncwarp();
       if (lane == 0) {
         rec.work = w;
-        rec.bh = bh;
+        rec.b = bh / p.st.H;
+        rec.h = bh - rec.b * p.st.H;
         rec.q_row = i * kBlk;
         if (has_approx) rec.desc[0] = ((uint32_t)j0 << 5) | kTileApprox;
         if (!item_has_tiles && end > first) rec.desc[first] |= kTileFirst;
@@ -341,10 +344,14 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
   uint32_t n_k = 0, n_v = 0, n_item = 0;
   Cursor cur_k, cur_v;
   PROF_DECL
-  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, int bh) {
+  // pooled = true: KC / mean-V operands, dense [B*H][Nk][d]; else q, k, v in the caller's layout
+  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, const Record* rec,
+                       bool pooled) {
     mbar_arrive_expect_tx(full, kTileBytes);
-    tma_load_3d(dst, tm, full, 0, row, bh);
-    tma_load_3d(dst + kHalfBytes, tm, full, 64, row, bh);
+    const bool rows_inner = pooled || p.rows_inner;
+    const int c1 = rows_inner ? row : rec->h, c2 = rows_inner ? rec->h : row;
+    tma_load_4d(dst, tm, full, 0, c1, c2, rec->b);
+    tma_load_4d(dst + kHalfBytes, tm, full, 64, c1, c2, rec->b);
   };
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
   bool k_end = false, have_k = false, ok = true;
@@ -362,14 +369,13 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
         have_k = true;
       }
       if (dk & kTileEnd) { have_k = false; continue; }
-      const int bh = cur_k.rec->bh;
       if (dk & kTileFirst) {
         // Q_i for this work item.  The slot frees when the previous item's last score GEMM
         // retires; until then serve the V side.
         const uint32_t par = (n_item & 1) ^ 1;
         if (n_k != n_v && !mbar_try_wait(&sm.q_empty, par)) break;
         if (!WAIT(&sm.q_empty, par, 2)) { ok = false; break; }                  // prof 2: Q slot busy
-        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, bh);
+        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, cur_k.rec, false);
         ++n_item;
         dk &= ~kTileFirst;
       }
@@ -378,7 +384,8 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
       if (!WAIT(&sm.k_empty[s], ((n_k / kKStages) & 1) ^ 1, 1)) { ok = false; break; }   // prof 1: K ring full
       {
         PROF_T0
-        load_tile((dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes, (int)(dk >> 5), bh);
+        load_tile((dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes, (int)(dk >> 5),
+                  cur_k.rec, (dk & kTileApprox) != 0);
         PROF_ADD(4)                                                                    // prof 4: issuing K copies
       }
       TRACE(n_k, 12);
@@ -404,7 +411,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     {
       PROF_T0
       load_tile((dv & kTileApprox) ? tm_vm : tm_v, &sm.v_full[s], sKV + (size_t)(kKStages + s) * kTileBytes,
-                (int)(dv >> 5), cur_v.rec->bh);
+                (int)(dv >> 5), cur_v.rec, (dv & kTileApprox) != 0);
       PROF_ADD(5)                                                                      // prof 5: issuing V copies
     }
     TRACE(n_v, 13);
@@ -682,7 +689,8 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     // ---- end of the work item: merge the two partial results, O_i = (w0 O0 + w1 O1) / (w0 l0 + w1 l1)
     const int q_row = cur.rec->q_row;
     const int q_rows = min(kBlk, p.N - q_row);
-    __nv_bfloat16* orow = p.out + ((size_t)cur.rec->bh * p.N + (size_t)(q_row + row)) * kD + h * kHalf;
+    __nv_bfloat16* orow = p.out + (size_t)cur.rec->b * (size_t)p.st.batch + (size_t)cur.rec->h * (size_t)p.st.head +
+                          (size_t)(q_row + row) * (size_t)p.st.row + h * kHalf;
     PROF_T0
     if (!(dsc & kTileEmptyItem)) {
       // the last P V of the item (one commit covers both halves)
@@ -818,14 +826,22 @@ cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __n
                              int32_t* counts, uint32_t* mask_out, cudaStream_t stream,
                              int* n_launches) {
   CUtensorMap tq, tk, tv, tkc, tvm;
-  if (!make_tmap_bf16_3d(&tq, q, p.BH, p.N, kD, kBlk) || !make_tmap_bf16_3d(&tk, k, p.BH, p.N, kD, kBlk) ||
-      !make_tmap_bf16_3d(&tv, v, p.BH, p.N, kD, kBlk) || !make_tmap_bf16_3d(&tkc, ws.kcb, p.BH, p.Nk, kD, kBlk) ||
-      !make_tmap_bf16_3d(&tvm, ws.vmb, p.BH, p.Nk, kD, kBlk))
+  bool rows_inner = true, pooled_inner = true;
+  auto user_map = [&](CUtensorMap* m, const void* base) {
+    return make_tmap_bf16_4d(m, base, p.B, p.H, p.N, kD, kBlk, p.st.row, p.st.head, p.st.batch, &rows_inner);
+  };
+  auto pooled_map = [&](CUtensorMap* m, const void* base) {      // dense [B][H][Nk][d]
+    return make_tmap_bf16_4d(m, base, p.B, p.H, p.Nk, kD, kBlk, kD, (long long)p.Nk * kD, (long long)p.H * p.Nk * kD,
+                             &pooled_inner);
+  };
+  if (!user_map(&tq, q) || !user_map(&tk, k) || !user_map(&tv, v) || !pooled_map(&tkc, ws.kcb) ||
+      !pooled_map(&tvm, ws.vmb) || !pooled_inner)
     return cudaErrorInvalidValue;
   Params prm{};
   prm.qbar = ws.qbar; prm.kc = ws.kc; prm.tau = tau; prm.out = out; prm.counts = counts; prm.mask_out = mask_out;
   prm.status = ws.status; prm.N = p.N; prm.Nq = p.Nq; prm.Nk = p.Nk; prm.total_work = p.BH * p.Nq;
   prm.mode = p.mode; prm.scale = p.scale; prm.forced = p.forced;
+  prm.st = p.st; prm.rows_inner = rows_inner ? 1 : 0;
 
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -21,7 +21,7 @@ struct alignas(16) Bf16x8 { __nv_bfloat162 v[4]; };
 template <int D>
 __global__ void __launch_bounds__(kPoolThreads)
 pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-            const __nv_bfloat16* __restrict__ v, WsPtrs ws, int N, int block_q, int block_k,
+            const __nv_bfloat16* __restrict__ v, WsPtrs ws, Strides st, int N, int block_q, int block_k,
             int Nq, int Nk, int first_kind) {
   constexpr int TPR = D / 8;                    // threads per row
   constexpr int RG = kPoolThreads / TPR;        // row groups
@@ -42,7 +42,7 @@ pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
   const __nv_bfloat16* src = (kind == 0) ? q : (kind == 1 ? k : v);
   const int row0 = blk * bs;
   const int nvalid = min(bs, N - row0);
-  const __nv_bfloat16* base = src + ((size_t)bh * N + row0) * D;
+  const __nv_bfloat16* base = src + st.base(bh) + (size_t)row0 * st.row;
 
   const int tc = threadIdx.x % TPR;             // which 8-channel group of the row
   const int g = threadIdx.x / TPR;              // row group
@@ -56,7 +56,7 @@ pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
     Bf16x8 x[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u)
-      x[u] = *reinterpret_cast<const Bf16x8*>(base + (size_t)(row + u * RG) * D + tc * 8);
+      x[u] = *reinterpret_cast<const Bf16x8*>(base + (size_t)(row + u * RG) * st.row + tc * 8);
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
@@ -67,7 +67,7 @@ pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
       }
   }
   for (; row < nvalid; row += RG) {
-    Bf16x8 x = *reinterpret_cast<const Bf16x8*>(base + (size_t)row * D + tc * 8);
+    Bf16x8 x = *reinterpret_cast<const Bf16x8*>(base + (size_t)row * st.row + tc * 8);
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float2 f = __bfloat1622float2(x.v[c]);
@@ -248,10 +248,10 @@ cudaError_t launch_pool(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
   const long long blocks = (long long)p.BH * ((q ? p.Nq : 0) + 2LL * p.Nk);
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   if (p.d == 128)
-    pool_kernel<128><<<(unsigned)blocks, kPoolThreads, 0, stream>>>(q, k, v, ws, p.N, p.block_q, p.block_k,
+    pool_kernel<128><<<(unsigned)blocks, kPoolThreads, 0, stream>>>(q, k, v, ws, p.st, p.N, p.block_q, p.block_k,
                                                                       p.Nq, p.Nk, first_kind);
   else
-    pool_kernel<64><<<(unsigned)blocks, kPoolThreads, 0, stream>>>(q, k, v, ws, p.N, p.block_q, p.block_k,
+    pool_kernel<64><<<(unsigned)blocks, kPoolThreads, 0, stream>>>(q, k, v, ws, p.st, p.N, p.block_q, p.block_k,
                                                                      p.Nq, p.Nk, first_kind);
   if (n_launches) *n_launches += 1;
   return cudaGetLastError();

@@ -23,16 +23,35 @@ inline EncodeTiledFn get_encode_tiled() {
   return fn;
 }
 
-// Tensor map over a contiguous bf16 [planes][rows][d] array: box = 64 channels x box_rows rows of
-// one plane, 128-byte swizzle, out-of-range rows read as zero (ragged last block).
-inline bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, int planes, int rows, int d, int box_rows) {
+// Tensor map over a bf16 tensor indexed (batch, head, row, channel) whose channels are contiguous
+// and whose other strides (in elements) are free: box = 64 channels x box_rows rows of one
+// (batch, head), 128-byte swizzle, out-of-range rows read as zero (ragged last block).
+// Dimensions are ordered by growing stride, as the encoder wants: rows_inner = true gives
+// coordinates (channel, row, head, batch), false gives (channel, head, row, batch).
+inline bool make_tmap_bf16_4d(CUtensorMap* map, const void* base, int B, int H, int rows, int d, int box_rows,
+                              long long row_stride, long long head_stride, long long batch_stride,
+                              bool* rows_inner) {
   EncodeTiledFn enc = get_encode_tiled();
   if (!enc) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)planes};
-  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2};   // bytes, dims 1 and 2
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  *rows_inner = row_stride <= head_stride;
+  cuuint64_t dims[4], strides[3];
+  cuuint32_t box[4];
+  dims[0] = (cuuint64_t)d;
+  box[0] = 64;
+  if (*rows_inner) {
+    dims[1] = (cuuint64_t)rows; dims[2] = (cuuint64_t)H;
+    strides[0] = (cuuint64_t)row_stride * 2; strides[1] = (cuuint64_t)head_stride * 2;
+    box[1] = (cuuint32_t)box_rows; box[2] = 1;
+  } else {
+    dims[1] = (cuuint64_t)H; dims[2] = (cuuint64_t)rows;
+    strides[0] = (cuuint64_t)head_stride * 2; strides[1] = (cuuint64_t)row_stride * 2;
+    box[1] = 1; box[2] = (cuuint32_t)box_rows;
+  }
+  dims[3] = (cuuint64_t)B;
+  strides[2] = (cuuint64_t)batch_stride * 2;
+  box[3] = 1;
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;

@@ -51,9 +51,14 @@ def unpack_mask(words: torch.Tensor, n_k: int) -> np.ndarray:
 
 
 def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, scale=0.0, want_mask=True,
-            tau_override=None, ws=None, estimator=0, forced=None):
-    """Run the fused forward through the C ABI; returns (out, counts, mask or None, ws)."""
+            tau_override=None, ws=None, estimator=0, forced=None, layout=0):
+    """Run the fused forward through the C ABI; returns (out, counts, mask or None, ws).
+
+    layout = SOL_LAYOUT_BNHD: q, k, v (and the returned out) are [B, N, H, d].
+    """
     B, H, N, d = q.shape
+    if layout == sb.SOL_LAYOUT_BNHD:
+        H, N = N, H
     if ws is None:
         ws = sb.make_workspace(B, H, N, d, block, block)
     out = torch.full_like(q, float("nan"))
@@ -62,7 +67,7 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
     if want_mask:
         mask_words = torch.zeros(B, H, ws.view.n_q_blocks, sb.mask_words(nk), dtype=torch.int32, device="cuda")
     sb.sol_attn_forward_ex(q, k, v, out, ws, block, block, threshold=beta, scale=scale, mode=mode, impl=impl,
-                           mask_out=mask_words, tau_override=tau_override, estimator=estimator,
+                           mask_out=mask_words, tau_override=tau_override, estimator=estimator, layout=layout,
                            forced_blocks=(None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.uint8)).cuda()))
     torch.cuda.synchronize()
     sb.sol_attn_bind_workspace(ws)

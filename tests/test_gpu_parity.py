@@ -311,3 +311,37 @@ def test_forced_exact_key_blocks(impl):
         ref = orc.dense_attention(synth.widen(bits[0][0, h], np.float64), synth.widen(bits[1][0, h], np.float64),
                                   synth.widen(bits[2][0, h], np.float64))
         assert (np.abs(hp.dev_to_f64(out2)[0, h] - ref) <= hp.out_bound(ref)).all()
+
+
+@pytest.mark.parametrize("impl,N,d,block", [("mma_sync", 1000, 64, 64), ("mma_sync", 1500, 128, 128),
+                                            ("tcgen05", 1500, 128, 128)])
+@pytest.mark.parametrize("mode_name", ["sol", "dense"])
+def test_token_major_layout(impl, N, d, block, mode_name):
+    """[B, N, H, d] inputs (heads interleaved per token) give bit for bit what [B, H, N, d] gives:
+    only addresses change, not the arithmetic; one head is also checked against the oracle."""
+    B, H = 2, 3
+    bits = _small_problem(31, B, H, N, d)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    mode = sb.SOL_MODE_SOL if mode_name == "sol" else sb.SOL_MODE_DENSE
+    out, counts, mask, _ = hp.run_gpu(q, k, v, block, 0.8, mode=mode, impl=_impl(impl))
+    qt, kt, vt = (x.permute(0, 2, 1, 3).contiguous() for x in (q, k, v))
+    out_t, counts_t, mask_t, _ = hp.run_gpu(qt, kt, vt, block, 0.8, mode=mode, impl=_impl(impl),
+                                            layout=sb.SOL_LAYOUT_BNHD)
+    assert out_t.shape == (B, N, H, d)
+    assert torch.equal(out_t.permute(0, 2, 1, 3).contiguous().view(torch.int16), out.view(torch.int16))
+    assert torch.equal(counts_t, counts)
+    assert np.array_equal(mask_t, mask)
+    if mode_name == "sol":
+        b, h = 1, 2
+        hp.check_head(synth.widen(bits[0][b, h], np.float64), synth.widen(bits[1][b, h], np.float64),
+                      synth.widen(bits[2][b, h], np.float64),
+                      hp.dev_to_f64(out_t.permute(0, 2, 1, 3).contiguous())[b, h], mask_t[b, h],
+                      counts_t[b, h].cpu().numpy(), block, 0.8)
+
+
+def test_layout_argument_is_validated():
+    bits = _small_problem(32, 1, 1, 256, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    ws = sb.make_workspace(1, 1, 256, 128, 128, 128)
+    with pytest.raises(RuntimeError):
+        sb.sol_attn_forward_ex(q, k, v, torch.empty_like(q), ws, 128, 128, threshold=0.5, layout=7)
