@@ -161,6 +161,62 @@ def threshold_diagonal(qbar, kc, beta: float, scale: float):
     return mu, sigma, _tau_from_stats(mu, sigma, beta)
 
 
+def route_topk(s_hat, k: int):
+    """Materialised top-k routing, the first baseline of the introduction: every query block keeps
+    the ``k`` key blocks with the highest proxy scores (ties go to the lower block index).
+
+    Returns (mask [N_q, N_k] bool, order [N_q, N_k] block indices by descending score, tau [N_q]).
+    ``tau`` is the threshold under which strict ``s_hat > tau`` reproduces the mask when the k-th and
+    (k+1)-th scores differ: their midpoint (-inf when every block is kept, +inf when none is)."""
+    s_hat = np.asarray(s_hat)
+    nq, nk = s_hat.shape
+    order = np.argsort(-s_hat, axis=1, kind="stable")
+    k = int(min(max(k, 0), nk))
+    mask = np.zeros((nq, nk), dtype=bool)
+    tau = np.empty(nq, dtype=s_hat.dtype)
+    for i in range(nq):
+        mask[i, order[i, :k]] = True
+        tau[i] = _cut_between(s_hat[i, order[i]], k)
+    return mask, order, tau
+
+
+def route_topp(s_hat, p: float):
+    """Materialised top-p routing, the second baseline of the introduction: per query block the key
+    blocks are taken in order of descending proxy score until their cumulative probability mass,
+    under the softmax of that row of proxy scores, reaches ``p``.
+
+    Returns (mask, order, tau, counts) as route_topk does; counts[i] is the number kept."""
+    s_hat = np.asarray(s_hat)
+    nq, nk = s_hat.shape
+    order = np.argsort(-s_hat, axis=1, kind="stable")
+    mask = np.zeros((nq, nk), dtype=bool)
+    tau = np.empty(nq, dtype=s_hat.dtype)
+    counts = np.zeros(nq, dtype=np.int64)
+    for i in range(nq):
+        row = s_hat[i, order[i]]
+        w = np.exp(row - row[0])
+        total = w.sum()
+        mass = 0.0
+        c = 0
+        while c < nk and mass < p * total:
+            mass += w[c]
+            c += 1
+        counts[i] = c
+        mask[i, order[i, :c]] = True
+        tau[i] = _cut_between(row, c)
+    return mask, order, tau, counts
+
+
+def _cut_between(sorted_desc, c: int):
+    """A cutoff that strict ``>`` turns into 'the first c of this descending row'."""
+    n = len(sorted_desc)
+    if c <= 0:
+        return np.inf
+    if c >= n:
+        return -np.inf
+    return 0.5 * (sorted_desc[c - 1] + sorted_desc[c])
+
+
 def select_blocks(s_hat, tau):
     """Eq. (4): boolean mask ``[N_q, N_k]``, True where ``s_ij > tau_i`` (strict)."""
     return s_hat > tau[:, None]

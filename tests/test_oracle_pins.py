@@ -371,3 +371,47 @@ def test_forced_blocks_and_diagonal_routing():
     np.testing.assert_allclose(rd.mu, base.mu, rtol=1e-12, atol=1e-14)
     v_k = np.var(base.kc, axis=0)                                   # numpy's own per-channel variance
     np.testing.assert_allclose(rd.sigma, np.sqrt((base.qbar ** 2) @ v_k) / math.sqrt(d), rtol=1e-10)
+
+
+# ----------------------------------------------------------------------------- materialised baselines
+def test_route_topk_is_the_k_largest():
+    """Top-k routing (introduction, limitation L1): brute force over all subsets of a small row."""
+    import itertools
+    rng = np.random.default_rng(5)
+    s = rng.standard_normal((6, 7))
+    for k in range(0, 8):
+        mask, order, tau = orc.route_topk(s, k)
+        assert (mask.sum(axis=1) == min(k, 7)).all()
+        for i in range(6):
+            best = max(itertools.combinations(range(7), min(k, 7)), key=lambda c: s[i, list(c)].sum())
+            assert set(np.flatnonzero(mask[i])) == set(best)
+            assert np.array_equal(s[i] > tau[i], mask[i])            # the equivalent threshold
+            assert (np.diff(s[i, order[i]]) <= 0).all()
+
+
+def test_route_topp_geometric_row_closed_form():
+    """Scores -j ln 2 give probabilities proportional to 2^-j: the mass of the c largest is
+    (1 - 2^-c) / (1 - 2^-N), so p = 0.9 keeps 4 blocks and p = 0.5 keeps 1 (N = 10)."""
+    n = 10
+    s = (-np.arange(n) * np.log(2.0))[None, :]
+    perm = np.random.default_rng(1).permutation(n)
+    sp = s[:, perm]
+    for p, want in [(0.9, 4), (0.5, 1), (0.5005, 2), (0.75, 2), (0.76, 3), (1.0, n)]:
+        mask, order, tau, counts = orc.route_topp(sp, p)
+        assert counts[0] == want, (p, counts)
+        assert set(perm[np.flatnonzero(mask[0])]) == set(range(want))
+        if want < n:
+            assert np.array_equal(sp[0] > tau[0], mask[0])
+
+
+def test_route_topp_uniform_row_and_budget_imbalance():
+    """Equal scores: each block carries 1/N of the mass, so ceil(p N) blocks are kept (lowest indices
+    first); a row dominated by one sink keeps a single block -- the budget imbalance the paper
+    attributes to top-p."""
+    n = 16
+    mask, order, tau, counts = orc.route_topp(np.zeros((1, n)), 0.3)
+    assert counts[0] == math.ceil(0.3 * n) and mask[0, :counts[0]].all()
+    s = np.zeros((1, n))
+    s[0, 11] = 12.0
+    mask, order, tau, counts = orc.route_topp(s, 0.9)
+    assert counts[0] == 1 and mask[0, 11]
