@@ -364,6 +364,29 @@ def main():
                           "speedup_vs_dense": ms_dense / ms_f, "one_over_density": 1.0 / dens})
         check_status()
 
+    # ---- routing latency: the thresholds of Eq. (4)/(5) (what the method needs before its single
+    #      pass) against the materialised baselines -- proxy map written to HBM, rows sorted,
+    #      top-k / top-p cut -- on the same pooled tensors
+    routing = None
+    if not args.no_sweep and world == 1 and wl.n_blocks <= 8192:
+        nb = wl.n_blocks
+        pmap = torch.empty(B, H, nb, nb, device="cuda")
+        order = torch.empty(B, H, nb, nb, dtype=torch.int32, device="cuda")
+        tau_b = torch.empty(B, H, nb, device="cuda")
+        cnt_b = torch.empty(B, H, nb, dtype=torch.int32, device="cuda")
+        k_blocks = max(1, int(round(args.density * nb)))
+        ms_thr = timed(lambda: sb.sol_attn_thresholds(B, H, N, d, wl.block, wl.block, beta), args.steps, 1)
+        ms_topk = timed(lambda: sb.sol_attn_route_materialized(ws.qbar, ws.kc, sb.SOL_ROUTE_TOPK, k_blocks, pmap,
+                                                               tau_b, order=order, counts=cnt_b), args.steps, 1)
+        ms_topp = timed(lambda: sb.sol_attn_route_materialized(ws.qbar, ws.kc, sb.SOL_ROUTE_TOPP, 0.9, pmap,
+                                                               tau_b, order=order, counts=cnt_b), args.steps, 1)
+        routing = {"thresholds_ms": ms_thr, "topk_ms": ms_topk, "topp_ms": ms_topp,
+                   "topk_over_thresholds": ms_topk / ms_thr, "topp_over_thresholds": ms_topp / ms_thr,
+                   "materialised_bytes": int(pmap.numel() * 4 + order.numel() * 4),
+                   "note": "thresholds: mean, covariance and tau kernels on pooled data (nothing of size Nq x Nk "
+                           "exists); baselines: proxy map + routing indices in HBM, k = %d blocks, p = 0.9" % k_blocks}
+        check_status()
+
     # ---- accuracy ablation on the image workload (small): error against dense attention of the
     #      full method vs keep-or-drop block-sparse attention under the SAME mask, and the spread of
     #      per-query-block densities (the counts output)
@@ -415,6 +438,7 @@ def main():
         "cpu_baseline": cpu,
         "sweep": sweep,
         "ablation": ablation,
+        "routing": routing,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

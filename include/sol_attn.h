@@ -113,6 +113,14 @@ sol_status_t sol_attn_pool(const void* q, const void* k, const void* v,
                            int B, int H, int N, int d, int block_q, int block_k,
                            float threshold, sol_stream_t stream);
 
+/* Threshold step alone (Eq. 5 pooled-key moments, Eq. 4 mu, sigma, tau) on the pooled tensors a
+ * previous sol_attn_pool / forward left in the bound workspace: re-thresholds the same q, k, v
+ * with another beta (density calibration, a per-step schedule) without reading them again.
+ * `scale` <= 0 selects 1/sqrt(d); `estimator` is SOL_EST_*.  Overwrites mu, sigma, tau in the
+ * workspace; a following sol_attn_forward_ex with skip_pool = 1 uses them. */
+sol_status_t sol_attn_thresholds(int B, int H, int N, int d, int block_q, int block_k, float threshold,
+                                 float scale, int estimator, sol_stream_t stream);
+
 /* Algorithm 1 end to end: the pooling pre-pass followed by the fused single-pass kernel
  * (on-the-fly thresholding, exact branch on routed blocks, approximate branch on the rest,
  * Eqs. 9-10), using the bound workspace.  Rows >= N of `out` do not exist and are never
@@ -198,6 +206,32 @@ sol_status_t sol_attn_thresholds_static(const float* qbar, const float* kc, int 
                                         int d, float scale, float threshold,
                                         float* mu, float* sigma, float* tau, sol_stream_t stream);
 size_t sol_attn_thresholds_static_max_floats(void);
+
+/* Materialised routing baselines: the two policies the paper compares its on-the-fly thresholding
+ * with (introduction, limitation L1; routing-latency figure).  The block proxy map of Eq. (3),
+ * s_ij = scale * Qbar_i . KC_j, is written to `proxy_map`, every row is read back and sorted, and
+ *   SOL_ROUTE_TOPK: the `param` (a block count, truncated to an integer, clamped to [0, Nk])
+ *                   highest-scoring key blocks of every query block are kept;
+ *   SOL_ROUTE_TOPP: blocks are kept in order of descending score until their share of the row's
+ *                   softmax mass, softmax_j(s_ij), reaches `param` = p in [0, 1].
+ * Equal scores are ordered by block index.
+ *
+ *   qbar, kc    device fp32 [B,H,Nq,d], [B,H,Nk,d]: pooled queries / keys (sol_attn_pool)
+ *   proxy_map   device fp32 [B,H,Nq,Nk], out: the materialised map (caller-owned, required)
+ *   order       device int32 [B,H,Nq,Nk] or NULL, out: block indices of each row by descending
+ *               score (the routing indices; the first counts[i] of them are the kept blocks)
+ *   tau         device fp32 [B,H,Nq], out: a cutoff equivalent to the selection -- the midpoint
+ *               between the last kept and the first dropped score (+inf: none kept, -inf: all) --
+ *               which sol_attn_forward_ex accepts as `tau_override`, so either policy can drive
+ *               the fused kernel
+ *   counts      device int32 [B,H,Nq] or NULL, out: kept blocks per query block
+ *
+ * Limits: Nk <= 8192 (a row is sorted in shared memory), d a multiple of 32; beyond them
+ * SOL_ERR_UNSUPPORTED_SHAPE and nothing is launched.  Allocates nothing; two kernels on `stream`. */
+enum { SOL_ROUTE_TOPK = 0, SOL_ROUTE_TOPP = 1 };
+sol_status_t sol_attn_route_materialized(const float* qbar, const float* kc, int B, int H, int Nq, int Nk,
+                                         int d, float scale, int policy, float param, float* proxy_map,
+                                         int32_t* order, float* tau, int32_t* counts, sol_stream_t stream);
 
 /* Number of kernels the library has launched since it was loaded (for launch accounting). */
 int64_t sol_attn_launch_count(void);

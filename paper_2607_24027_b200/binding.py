@@ -29,12 +29,14 @@ SOL_MODE_SOL, SOL_MODE_DENSE, SOL_MODE_EXACT_ONLY = 0, 1, 2
 SOL_IMPL_AUTO, SOL_IMPL_TCGEN05, SOL_IMPL_MMA_SYNC = 0, 1, 2
 SOL_EST_MOMENTS, SOL_EST_DIAGONAL = 0, 1
 SOL_LAYOUT_BHND, SOL_LAYOUT_BNHD = 0, 1
+SOL_ROUTE_TOPK, SOL_ROUTE_TOPP = 0, 1
 
 EXPORTS = [
     "sol_attn_status_string", "sol_attn_workspace_bytes", "sol_attn_workspace_view",
     "sol_attn_bind_workspace", "sol_attn_pool", "sol_attn_forward", "sol_attn_dense",
     "sol_attn_forward_ex", "sol_attn_forward_host", "sol_attn_read_device_status",
     "sol_attn_launch_count", "sol_attn_thresholds_static", "sol_attn_thresholds_static_max_floats",
+    "sol_attn_route_materialized", "sol_attn_thresholds",
 ]
 
 
@@ -88,6 +90,8 @@ def lib() -> ctypes.CDLL:
     L.sol_attn_bind_workspace.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
     L.sol_attn_pool.restype = ctypes.c_int32
     L.sol_attn_pool.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 6 + [ctypes.c_float, ctypes.c_void_p]
+    L.sol_attn_thresholds.restype = ctypes.c_int32
+    L.sol_attn_thresholds.argtypes = [ctypes.c_int] * 6 + [ctypes.c_float] * 2 + [ctypes.c_int, ctypes.c_void_p]
     L.sol_attn_forward.restype = ctypes.c_int32
     L.sol_attn_forward.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 6 + [ctypes.c_float, ctypes.c_void_p]
     L.sol_attn_dense.restype = ctypes.c_int32
@@ -105,6 +109,10 @@ def lib() -> ctypes.CDLL:
                                             [ctypes.c_void_p] * 4
     L.sol_attn_thresholds_static_max_floats.restype = ctypes.c_size_t
     L.sol_attn_thresholds_static_max_floats.argtypes = []
+    L.sol_attn_route_materialized.restype = ctypes.c_int32
+    L.sol_attn_route_materialized.argtypes = [ctypes.c_void_p] * 2 + [ctypes.c_int] * 5 + [ctypes.c_float, ctypes.c_int,
+                                                                                           ctypes.c_float] + \
+                                             [ctypes.c_void_p] * 5
     _lib = L
     return L
 
@@ -259,6 +267,32 @@ def sol_attn_thresholds_static(qbar, kc, threshold, mu, sigma, tau, scale=0.0, s
     _check(lib().sol_attn_thresholds_static(_ptr(qbar), _ptr(kc), B, H, Nq, Nk, d, float(scale), float(threshold),
                                             _ptr(mu), _ptr(sigma), _ptr(tau), _stream(stream)),
            "sol_attn_thresholds_static")
+
+
+def sol_attn_thresholds(B, H, N, d, block_q, block_k, threshold, scale=0.0, estimator=SOL_EST_MOMENTS, stream=None):
+    """Recompute mu, sigma, tau in the bound workspace from the pooled tensors already there."""
+    _check(lib().sol_attn_thresholds(B, H, N, d, block_q, block_k, float(threshold), float(scale), int(estimator),
+                                     _stream(stream)), "sol_attn_thresholds")
+
+
+def sol_attn_route_materialized(qbar, kc, policy, param, proxy_map, tau, order=None, counts=None, scale=0.0,
+                                stream=None):
+    """Top-k / top-p routing over a proxy map written to ``proxy_map`` (fp32 [B, H, Nq, Nk]); fills ``tau``
+    (fp32 [B, H, Nq], usable as ``tau_override``), optionally ``order`` (int32 [B, H, Nq, Nk]) and ``counts``."""
+    B, H, Nq, d = (int(x) for x in qbar.shape)
+    Nk = int(kc.shape[2])
+    for t in (qbar, kc, proxy_map, tau):
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("expected contiguous CUDA fp32 tensors")
+    for t in (order, counts):
+        if t is not None and (t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("expected contiguous CUDA int32 tensors")
+    if proxy_map.numel() != B * H * Nq * Nk or tau.numel() != B * H * Nq:
+        raise ValueError("proxy_map / tau have the wrong size")
+    _check(lib().sol_attn_route_materialized(_ptr(qbar), _ptr(kc), B, H, Nq, Nk, d, float(scale), int(policy),
+                                             float(param), _ptr(proxy_map), _ptr(order), _ptr(tau), _ptr(counts),
+                                             _stream(stream)),
+           "sol_attn_route_materialized")
 
 
 def sol_attn_thresholds_static_max_floats() -> int:

@@ -127,6 +127,23 @@ sol_status_t sol_attn_pool(const void* q, const void* k, const void* v, int B, i
   return run_pool(p, q, k, v, g_bound.ws, static_cast<cudaStream_t>(stream));
 }
 
+sol_status_t sol_attn_thresholds(int B, int H, int N, int d, int block_q, int block_k, float threshold, float scale,
+                                 int estimator, sol_stream_t stream) {
+  sol_status_t s = check_shape(B, H, N, d, block_q, block_k, false);
+  if (s != SOL_OK) return s;
+  if (std::isnan(threshold) || std::isnan(scale) || std::isinf(scale)) return SOL_ERR_INVALID_ARG;
+  if (estimator != SOL_EST_MOMENTS && estimator != SOL_EST_DIAGONAL) return SOL_ERR_INVALID_ARG;
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  if (g_bound.bytes < sol_attn_workspace_bytes(B, H, N, d, block_q, block_k)) return SOL_ERR_WORKSPACE;
+  if ((s = check_arch()) != SOL_OK) return s;
+  const sol::Problem p = make_problem(B, H, N, d, block_q, block_k, threshold, scale, SOL_MODE_SOL, estimator);
+  const sol::WsPtrs ws = sol::make_ptrs(g_bound.ws, sol::make_layout(p.BH, p.Nq, p.Nk, p.d));
+  int n = 0;
+  const cudaError_t e = sol::launch_thresholds(p, ws, static_cast<cudaStream_t>(stream), &n);
+  g_launches += n;
+  return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+}
+
 sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
   if (!a) return SOL_ERR_INVALID_ARG;
   sol_status_t s = check_shape(a->B, a->H, a->N, a->d, a->block_q, a->block_k, true);
