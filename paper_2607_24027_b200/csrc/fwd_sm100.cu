@@ -139,9 +139,11 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_FLUSH(role) prof.flush(role)
 #define PROF_ACC(slot) (&prof.v[slot])
 // timeline of a few tiles of CTA 0: [tile][event] = clock64()
-constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 32;
+constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 80;
 __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
+// per-warp phases of the softmax role: events 32 + 6 * warp + k
+#define WTRACE(k) do { if (lane == 0) TRACE(g, 32 + (4 * h + warp_in_group) * 6 + (k)); } while (0)
 #define PROF_T0 const long long prof_t0 = clock64();
 #define PROF_ADD(slot) prof.v[slot] += clock64() - prof_t0;
 #else
@@ -151,6 +153,7 @@ __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #define PROF_FLUSH(role)
 #define PROF_ACC(slot) nullptr
 #define TRACE(tile, evt)
+#define WTRACE(k)
 #define PROF_T0
 #define PROF_ADD(slot)
 #endif
@@ -584,12 +587,14 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
       tc_fence_after();
       if (row == 0) TRACE(g, 6 + 3 * h);
+      WTRACE(0);
       // ---- this group's half row of S (64 fp32) into registers with one wait
       uint32_t sr[kHalf];
       PROF_T0
       tmem_ld_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
       tmem_ld_32x32b_x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
       tmem_ld_wait();
+      WTRACE(1);
       PROF_ADD(7)                                                                      // prof 7: loading S
       if (general) {
         // bring the rare tiles (approximate chunk, ragged last block) to the common form
@@ -645,6 +650,7 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         l *= f;
         m_used = m_new;
       }
+      WTRACE(2);
       // ---- P = exp2(sl2 * S - m) (scaling and row sum as packed fp32 pairs); P (bf16) back to
       //      TMEM over the start of the half
       {
@@ -672,11 +678,14 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       }
       PROF_ADD(8)                                                                      // prof 8: load + arithmetic
       if (row == 0) TRACE(g, 7 + 3 * h);
+      WTRACE(3);
       tmem_st_wait();
+      WTRACE(4);
       tc_fence_before();
       mbar_arrive(&sm.p_full[h][b]);
       if (row == 0) TRACE(g, 8 + 3 * h);
       if (lane == 0) TRACE(g, 16 + 4 * h + warp_in_group);
+      WTRACE(5);
       PROF_ADD(9)                                                                      // prof 9: whole tile
 #ifdef SOL_PROFILE
       if (approx) { prof.v[10] += clock64() - prof_t0; ++prof.v[0]; }                  // prof 10 / 0: approximate tiles: cycles / count
