@@ -166,10 +166,15 @@ typedef struct {
 } sol_attn_args;
 sol_status_t sol_attn_forward_ex(const sol_attn_args* args /* host */);
 
-/* End-to-end convenience for callers whose tensors live in HOST memory (pinned memory makes
- * the copies asynchronous): copies hq, hk, hv into the caller's device staging buffers dq, dk,
- * dv, runs sol_attn_forward with the bound workspace, copies dout into hout, all on `stream`.
- * Does not synchronise. */
+/* End-to-end convenience for callers whose tensors live in HOST memory ([B,H,N,d] layout;
+ * pinned memory makes the copies asynchronous).  Heads are independent, so the call is cut into
+ * groups of heads (about 64 MB per tensor) and pipelined: the kernels of one group run on
+ * `stream` while the next group's q, k, v are copied into the caller's device staging buffers
+ * dq, dk, dv and the previous group's part of dout is copied to hout.  The copies use two streams
+ * that the library creates on first use (per device, kept until the process ends); `stream` is
+ * made to wait for the last copy back, so work queued on it afterwards sees hout complete.
+ * Uses the bound workspace and counts.  Does not synchronise the host.  The environment variable
+ * SOL_ATTN_HOST_GROUP_BYTES, when set to a positive number, replaces the 64 MB group size. */
 sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* hv, void* hout,
                                    void* dq, void* dk, void* dv, void* dout,
                                    int B, int H, int N, int d, int block_q, int block_k,

@@ -1,7 +1,9 @@
 // C ABI of the Sol-Attn CUDA path: argument validation, workspace bookkeeping, launches.
 #include <atomic>
+#include <mutex>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -16,6 +18,26 @@ Bound g_bound;
 std::atomic<int64_t> g_launches{0};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Two copy streams per device for the host-buffer entry point, made on first use and kept for the
+// life of the process (streams are host-side objects; no device memory is involved).
+constexpr int kMaxDevices = 64;
+std::mutex g_stream_mu;
+cudaStream_t g_copy_in[kMaxDevices] = {nullptr}, g_copy_out[kMaxDevices] = {nullptr};
+
+sol_status_t copy_streams(cudaStream_t* in, cudaStream_t* out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return SOL_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lock(g_stream_mu);
+  if (!g_copy_in[dev]) {
+    if (cudaStreamCreateWithFlags(&g_copy_in[dev], cudaStreamNonBlocking) != cudaSuccess) return SOL_ERR_CUDA;
+    if (cudaStreamCreateWithFlags(&g_copy_out[dev], cudaStreamNonBlocking) != cudaSuccess) return SOL_ERR_CUDA;
+  }
+  *in = g_copy_in[dev];
+  *out = g_copy_out[dev];
+  return SOL_OK;
+}
 
 sol_status_t check_arch() {
   int dev = 0;
@@ -144,7 +166,8 @@ sol_status_t sol_attn_thresholds(int B, int H, int N, int d, int block_q, int bl
   return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
 
-sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
+// keep_status: a later piece of one logical call must not wipe the device status of an earlier one
+static sol_status_t forward_impl(const sol_attn_args* a, bool keep_status) {
   if (!a) return SOL_ERR_INVALID_ARG;
   sol_status_t s = check_shape(a->B, a->H, a->N, a->d, a->block_q, a->block_k, true);
   if (s != SOL_OK) return s;
@@ -170,7 +193,10 @@ sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
   cudaStream_t stream = static_cast<cudaStream_t>(a->stream);
   const sol::WsLayout lay = sol::make_layout(p.BH, p.Nq, p.Nk, p.d);
   const sol::WsPtrs ws = sol::make_ptrs(a->workspace, lay);
-  if (cudaMemsetAsync(ws.status, 0, sizeof(int32_t) * sol::kStatusWords, stream) != cudaSuccess) return SOL_ERR_CUDA;
+  const int first_word = keep_status ? sol::kStatusTileCounter : 0;
+  if (cudaMemsetAsync(ws.status + first_word, 0, sizeof(int32_t) * (sol::kStatusWords - first_word), stream) !=
+      cudaSuccess)
+    return SOL_ERR_CUDA;
   if (p.mode != SOL_MODE_DENSE && !a->skip_pool) {
     s = run_pool(p, a->q, a->k, a->v, a->workspace, stream);
     if (s != SOL_OK) return s;
@@ -187,6 +213,8 @@ sol_status_t sol_attn_forward_ex(const sol_attn_args* a) {
   g_launches += n;
   return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
+
+sol_status_t sol_attn_forward_ex(const sol_attn_args* a) { return forward_impl(a, false); }
 
 sol_status_t sol_attn_forward(const void* q, const void* k, const void* v, void* out, int B, int H, int N,
                               int d, int block_q, int block_k, float threshold, sol_stream_t stream) {
@@ -219,14 +247,72 @@ sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* h
   if (!hq || !hk || !hv || !hout || !dq || !dk || !dv || !dout) return SOL_ERR_INVALID_ARG;
   sol_status_t s = check_shape(B, H, N, d, block_q, block_k, true);
   if (s != SOL_OK) return s;
-  const size_t bytes = (size_t)B * H * N * d * 2;
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  if (g_bound.bytes < sol_attn_workspace_bytes(B, H, N, d, block_q, block_k)) return SOL_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(dq, hq, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
-  if (cudaMemcpyAsync(dk, hk, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
-  if (cudaMemcpyAsync(dv, hv, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SOL_ERR_CUDA;
-  s = sol_attn_forward(dq, dk, dv, dout, B, H, N, d, block_q, block_k, threshold, stream);
-  if (s != SOL_OK) return s;
-  if (cudaMemcpyAsync(hout, dout, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SOL_ERR_CUDA;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  if ((s = copy_streams(&s_in, &s_out)) != SOL_OK) return s;
+
+  // Heads are independent, so the call is cut into groups of heads and pipelined: while the
+  // kernels work on one group (on the caller's stream), the next group's q, k, v travel to the
+  // device on one copy stream and the previous group's output travels back on another.
+  const int BH = B * H, Nq = sol::ceil_div(N, block_q);
+  const size_t head_bytes = (size_t)N * d * 2;
+  size_t want = size_t(64) << 20;                            // about 64 MB per tensor and group
+  if (const char* env = getenv("SOL_ATTN_HOST_GROUP_BYTES")) {    // tuning / test knob
+    const long long v = atoll(env);
+    if (v > 0) want = (size_t)v;
+  }
+  int per = (int)((want + head_bytes - 1) / head_bytes);
+  if (per < 1) per = 1;
+  if (per > BH) per = BH;
+  auto fail = [](cudaEvent_t a, cudaEvent_t b) {
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    return SOL_ERR_CUDA;
+  };
+  // copies must not overtake work already queued on the caller's stream (it may still use dq...)
+  cudaEvent_t e0 = nullptr;
+  if (cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
+  if (cudaEventRecord(e0, st) != cudaSuccess || cudaStreamWaitEvent(s_in, e0, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(s_out, e0, 0) != cudaSuccess)
+    return fail(e0, nullptr);
+  cudaEventDestroy(e0);
+  bool first = true;
+  for (int h0 = 0; h0 < BH; h0 += per) {
+    const int nh = (BH - h0 < per) ? BH - h0 : per;
+    const size_t off = (size_t)h0 * head_bytes, bytes = (size_t)nh * head_bytes;
+    auto at = [off](const void* p) { return static_cast<const char*>(p) + off; };
+    auto at_w = [off](void* p) { return static_cast<char*>(p) + off; };
+    cudaEvent_t e_in = nullptr, e_done = nullptr;
+    if (cudaEventCreateWithFlags(&e_in, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&e_done, cudaEventDisableTiming) != cudaSuccess) return fail(e_in, nullptr);
+    if (cudaMemcpyAsync(at_w(dq), at(hq), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(dk), at(hk), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(dv), at(hv), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaEventRecord(e_in, s_in) != cudaSuccess || cudaStreamWaitEvent(st, e_in, 0) != cudaSuccess)
+      return fail(e_in, e_done);
+    sol_attn_args a{};
+    a.q = at_w(dq); a.k = at_w(dk); a.v = at_w(dv); a.out = at_w(dout);
+    a.B = 1; a.H = nh; a.N = N; a.d = d; a.block_q = block_q; a.block_k = block_k;
+    a.threshold = threshold; a.scale = 0.f; a.mode = SOL_MODE_SOL; a.impl = SOL_IMPL_AUTO;
+    a.workspace = g_bound.ws; a.workspace_bytes = g_bound.bytes;
+    a.counts = g_bound.counts ? g_bound.counts + (size_t)h0 * Nq : nullptr;
+    a.stream = stream;
+    s = forward_impl(&a, !first);
+    first = false;
+    if (s != SOL_OK) { fail(e_in, e_done); return s; }
+    if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(s_out, e_done, 0) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(hout), at(dout), bytes, cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
+      return fail(e_in, e_done);
+    cudaEventDestroy(e_in);
+    cudaEventDestroy(e_done);
+  }
+  // the caller's stream ends where the last copy back ends
+  cudaEvent_t e1 = nullptr;
+  if (cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
+  if (cudaEventRecord(e1, s_out) != cudaSuccess || cudaStreamWaitEvent(st, e1, 0) != cudaSuccess) return fail(e1, nullptr);
+  cudaEventDestroy(e1);
   return SOL_OK;
 }
 

@@ -246,6 +246,30 @@ def test_bound_entry_points_and_host_path():
         assert (np.abs(hp.dev_to_f64(dense)[0, h] - refd) <= hp.out_bound(refd)).all()
 
 
+def test_host_path_pipelined_over_head_groups(monkeypatch):
+    """The host-buffer entry point cut into several groups of heads (copies on their own streams,
+    kernels on the caller's) returns what one device-resident call returns, counts included."""
+    B, H, N, d, block = 2, 5, 700, 128, 128
+    bits = _small_problem(33, B, H, N, d)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    ref, counts_ref, _, _ = hp.run_gpu(q, k, v, block, 0.7)
+    ws = sb.make_workspace(B, H, N, d, block, block)
+    sb.sol_attn_bind_workspace(ws)
+    hq, hk, hv = (torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory() for x in bits)
+    dq, dk, dv, dout = (torch.empty_like(q) for _ in range(4))
+    for group_bytes in (N * d * 2 * 3, N * d * 2, 1 << 30):            # 3 heads, 1 head, everything at once
+        monkeypatch.setenv("SOL_ATTN_HOST_GROUP_BYTES", str(group_bytes))
+        hout = torch.zeros_like(hq).pin_memory()
+        ws.counts.fill_(-1)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            sb.sol_attn_forward_host(hq, hk, hv, hout, dq, dk, dv, dout, block, block, 0.7)
+            side.synchronize()
+        assert torch.equal(hout, ref.view(torch.int16).cpu()), group_bytes
+        assert torch.equal(ws.counts, counts_ref)
+        assert sb.sol_attn_read_device_status() == sb.SOL_OK
+
+
 @pytest.mark.parametrize("impl", IMPLS_128)
 @pytest.mark.parametrize("jump", [3.0, 6.0])
 def test_reference_maximum_jumps(impl, jump):
