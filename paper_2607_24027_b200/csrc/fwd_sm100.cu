@@ -139,7 +139,10 @@ __device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volati
 #define PROF_FLUSH(role) prof.flush(role)
 #define PROF_ACC(slot) (&prof.v[slot])
 // timeline of a few tiles of CTA 0: [tile][event] = clock64()
-constexpr int kTraceFirst = 40, kTraceTiles = 16, kTraceEvents = 80;
+#ifndef SOL_TRACE_FIRST
+#define SOL_TRACE_FIRST 40
+#endif
+constexpr int kTraceFirst = SOL_TRACE_FIRST, kTraceTiles = 16, kTraceEvents = 80;
 __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
 // per-warp phases of the softmax role: events 32 + 6 * warp + k
