@@ -369,3 +369,43 @@ def test_layout_argument_is_validated():
     ws = sb.make_workspace(1, 1, 256, 128, 128, 128)
     with pytest.raises(RuntimeError):
         sb.sol_attn_forward_ex(q, k, v, torch.empty_like(q), ws, 128, 128, threshold=0.5, layout=7)
+
+
+# ----------------------------------------------------------------------------- degenerate inputs
+@pytest.mark.parametrize("impl", IMPLS_128)
+def test_degenerate_inputs(impl):
+    """Cases in which the method's statistics collapse: zero queries and keys (every logit 0, sigma = 0,
+    uniform attention), keys constant within each block (the proxy term is exact, so the output is
+    dense attention whatever beta selects), a single token, exactly one block."""
+    rng = np.random.default_rng(7)
+    d, block = 128, 128
+    # (a) zero q and k: out = mean of v over all tokens, nothing NaN, counts in range
+    N = 700
+    z = np.zeros((1, 1, N, d), dtype=np.float32)
+    vb = synth.f32_to_bf16_bits(rng.standard_normal((1, 1, N, d)).astype(np.float32))
+    zb = synth.f32_to_bf16_bits(z)
+    q, k, v = hp.to_dev(zb), hp.to_dev(zb), hp.to_dev(vb)
+    out, counts, mask, _ = hp.run_gpu(q, k, v, block, 0.5, impl=_impl(impl))
+    want = synth.widen(vb[0, 0], np.float64).mean(axis=0)
+    got = hp.dev_to_f64(out)[0, 0]
+    assert np.isfinite(got).all()
+    assert np.abs(got - want[None, :]).max() <= 1e-2
+    c = counts.cpu().numpy()
+    assert (c >= 0).all() and (c <= 6).all()
+    # (b) keys constant within each block: Sol-Attn equals dense attention for every beta
+    N = 900
+    nb = (N + block - 1) // block
+    kconst = np.repeat(rng.standard_normal((nb, d)).astype(np.float32), block, axis=0)[:N]
+    qf = rng.standard_normal((N, d)).astype(np.float32)
+    vf = rng.standard_normal((N, d)).astype(np.float32)
+    bits = [synth.f32_to_bf16_bits(x[None, None]) for x in (qf, kconst, vf)]
+    ref = orc.dense_attention(*(synth.widen(x[0, 0], np.float64) for x in bits))
+    for beta in (-0.5, 0.8, math.inf):
+        out, _, _, _ = hp.run_gpu(*(hp.to_dev(x) for x in bits), block, beta, impl=_impl(impl))
+        got = hp.dev_to_f64(out)[0, 0]
+        assert (np.abs(got - ref) <= hp.out_bound(ref)).all(), beta
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= hp.REL_L2
+    # (c) one token; exactly one full block; more (batch, head) pairs than tokens per block
+    for B, H, N in ((1, 1, 1), (1, 2, 128), (3, 7, 200)):
+        bits = _small_problem(50 + N, B, H, N, d)
+        _check_all_heads(bits, block, 0.4, _impl(impl))
