@@ -685,7 +685,8 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       tmem_st_wait();
       WTRACE(4);
       tc_fence_before();
-      mbar_arrive(&sm.p_full[h][b]);
+      __syncwarp();                                  // one arrival per warp: 4 instead of 128 on the barrier
+      if (lane == 0) mbar_arrive(&sm.p_full[h][b]);
       if (row == 0) TRACE(g, 8 + 3 * h);
       if (lane == 0) TRACE(g, 16 + 4 * h + warp_in_group);
       WTRACE(5);
@@ -782,8 +783,8 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm.s_full[b], 1);
       mbar_init(&sm.pv_done[b], 1);
-      mbar_init(&sm.p_full[0][b], 128);
-      mbar_init(&sm.p_full[1][b], 128);
+      mbar_init(&sm.p_full[0][b], 4);
+      mbar_init(&sm.p_full[1][b], 4);
     }
     mbar_init(&sm.x_full, 256); mbar_init(&sm.x_done, 256);
     mbar_init(&sm.kc_full[0], 1); mbar_init(&sm.kc_full[1], 1);
