@@ -164,6 +164,9 @@ typedef struct {
                                                    batches and heads; counts include them         */
   int32_t layout;                               /* SOL_LAYOUT_* of q, k, v and out (0 = [B,H,N,d]) */
 } sol_attn_args;
+/* Everything sol_attn_forward_ex enqueues is ordinary work on `stream` (a memset of the status words
+ * and kernels), so the call may be captured into a CUDA graph and replayed; sol_attn_forward_host may
+ * not (it creates events and uses streams of its own). */
 sol_status_t sol_attn_forward_ex(const sol_attn_args* args /* host */);
 
 /* End-to-end convenience for callers whose tensors live in HOST memory ([B,H,N,d] layout;

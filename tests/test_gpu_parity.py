@@ -409,3 +409,33 @@ def test_degenerate_inputs(impl):
     for B, H, N in ((1, 1, 1), (1, 2, 128), (3, 7, 200)):
         bits = _small_problem(50 + N, B, H, N, d)
         _check_all_heads(bits, block, 0.4, _impl(impl))
+
+
+@pytest.mark.parametrize("impl", IMPLS_128)
+def test_cuda_graph_capture_and_replay(impl):
+    """The whole call (status reset, pooling, thresholds, fused kernel) is plain stream work: it can
+    be captured into a CUDA graph and replayed, with new input values in the same buffers."""
+    bits = _small_problem(61, 1, 2, 1100, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    ws = sb.make_workspace(1, 2, 1100, 128, 128, 128)
+    out = torch.empty_like(q)
+    eager, counts_eager, _, _ = hp.run_gpu(q, k, v, 128, 0.6, impl=_impl(impl), want_mask=False)
+    sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.6, impl=_impl(impl))   # warm-up outside capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.6, impl=_impl(impl))
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), eager.view(torch.int16))
+    assert torch.equal(ws.counts, counts_eager)
+    # new values in the same buffers: the replay recomputes everything
+    bits2 = _small_problem(62, 1, 2, 1100, 128)
+    for dst, src in zip((q, k, v), bits2):
+        dst.copy_(hp.to_dev(src))
+    graph.replay()
+    torch.cuda.synchronize()
+    eager2, counts2, _, _ = hp.run_gpu(q, k, v, 128, 0.6, impl=_impl(impl), want_mask=False)
+    assert torch.equal(out.view(torch.int16), eager2.view(torch.int16))
+    assert torch.equal(ws.counts, counts2)
