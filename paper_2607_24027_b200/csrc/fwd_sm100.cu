@@ -459,7 +459,7 @@ __device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo) {
   return ((uint64_t)hi << 32) | lo;
 }
 
-// S_b = Q K^T (warp 10, one thread)
+// S_b = Q K^T (warp 10)
 __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV, uint32_t tmem) {
   const uint32_t idesc_qk = make_idesc_bf16(kBlk, kBlk, false, false);
   const uint32_t q_lo = (smem_addr(sQ) >> 4) | (1u << 16);
@@ -468,14 +468,18 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
   uint32_t slot = 0, slot_parity = 0;          // ring position of K(g)
   Cursor cur;
   PROF_DECL
-  auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
+  // The whole warp runs this role in lockstep and one elected lane issues: with warp-uniform control
+  // flow and operands the compiler keeps descriptors and addresses in uniform registers, where the
+  // MMA instruction wants them, instead of moving them over from a single divergent lane's registers.
+  const bool leader = elect_one();
+  auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
+    const uint32_t dsc = __shfl_sync(0xffffffffu, next_desc(sm, cur, PROF_ACC(0), release), 0);                    // prof 0: no record yet
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) {                         // every MMA that reads Q_i has been issued
-      if (!(dsc & kTileEmptyItem)) mma_commit(&sm.q_empty);
+      if (!(dsc & kTileEmptyItem) && leader) mma_commit(&sm.q_empty);
       continue;
     }
     if (dsc & kTileFirst) {
@@ -500,32 +504,35 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
         const uint32_t off = ((ks / 4) * kHalfBytes + (ks % 4) * 32) >> 4;
-        mma_ss(d_tmem, desc_from_lo(q_lo + off), desc_from_lo(k_lo + off), idesc_qk, ks > 0);
+        const uint64_t da = desc_from_lo(q_lo + off), db = desc_from_lo(k_lo + off);
+        if (leader) mma_ss(d_tmem, da, db, idesc_qk, ks > 0);
       }
-      mma_commit(&sm.k_empty[slot]);
-      mma_commit(&sm.s_full[b]);
+      if (leader) {
+        mma_commit(&sm.k_empty[slot]);
+        mma_commit(&sm.s_full[b]);
+      }
       PROF_ADD(6)                                                                      // prof 6: issuing Q K^T
     }
     TRACE(g, 1);
     ++g;
     if (++slot == kKStages) { slot = 0; slot_parity ^= 1; }
   }
-  if (!ok) flag_abort(sm, p, 300);
-  PROF_FLUSH(2);
+  if (!ok && leader) flag_abort(sm, p, 300);
+  if (leader) PROF_FLUSH(2);
 }
 
-// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11, one thread); the fixed-reference variant has
-// one accumulator and P in its own columns
+// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11)
 __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uint32_t tmem) {
   const uint32_t idesc_pv = make_idesc_bf16(kBlk, kD, false, true);
   const uint32_t kv_lo = (smem_addr(sKV + kKStages * kTileBytes) >> 4) | ((uint32_t)(kHalfBytes >> 4) << 16);
   uint32_t g = 0;
   uint32_t slot = 0, slot_parity = 0;          // ring position of V(g)
   Cursor cur;
-  auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
+  const bool leader = elect_one();             // warp-uniform role, one issuing lane (see mma_qk_role)
+  auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, nullptr, release);
+    const uint32_t dsc = __shfl_sync(0xffffffffu, next_desc(sm, cur, nullptr, release), 0);
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) continue;
@@ -544,17 +551,20 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
         const uint32_t d_o = tmem + kTmemO + h * kD;
         const uint32_t a_p = tmem + kTmemS + b * kBlk + h * kHalf + ks * 8;
         const uint32_t acc = ks > 0 ? 1u : acc_first;
-        mma_ts(d_o, a_p, desc_from_lo(v_lo + ((h * (kHalf * 128) + ks * 2048) >> 4)), idesc_pv, acc);
+        const uint64_t dv = desc_from_lo(v_lo + ((h * (kHalf * 128) + ks * 2048) >> 4));
+        if (leader) mma_ts(d_o, a_p, dv, idesc_pv, acc);
       }
     }
     if (!ok) break;
-    mma_commit(&sm.v_empty[slot]);
-    mma_commit(&sm.pv_done[b]);
+    if (leader) {
+      mma_commit(&sm.v_empty[slot]);
+      mma_commit(&sm.pv_done[b]);
+    }
     TRACE(g, 5);
     ++g;
     if (++slot == kVStages) { slot = 0; slot_parity ^= 1; }
   }
-  if (!ok) flag_abort(sm, p, 301);
+  if (!ok && leader) flag_abort(sm, p, 301);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -807,9 +817,9 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == kWarpProducer) {
     if (lane == 0) producer_role(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
   } else if (warp == kWarpQK) {
-    if (lane == 0) mma_qk_role(sm, p, sQ, sKV, tmem);
+    mma_qk_role(sm, p, sQ, sKV, tmem);
   } else {
-    if (lane == 0) mma_pv_role(sm, p, sKV, tmem);
+    mma_pv_role(sm, p, sKV, tmem);
   }
   tc_fence_before();
   __syncthreads();
