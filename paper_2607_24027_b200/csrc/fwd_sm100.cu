@@ -475,7 +475,7 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
   auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = __shfl_sync(0xffffffffu, next_desc(sm, cur, PROF_ACC(0), release), 0);                    // prof 0: no record yet
+    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) {                         // every MMA that reads Q_i has been issued
@@ -532,7 +532,7 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
   auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = __shfl_sync(0xffffffffu, next_desc(sm, cur, nullptr, release), 0);
+    const uint32_t dsc = next_desc(sm, cur, nullptr, release);
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) continue;
