@@ -7,13 +7,14 @@
 //                      pooled keys in chunks of 128 blocks.  For every block it evaluates the
 //                      proxy s_ij = scale * Qbar_i . KC_j (Eq. 3) in fp32 and compares it with
 //                      tau_i (Eq. 4).  The decision only ever lives in a small shared-memory
-//                      record (selected list + per-column bias); nothing of the proxy map goes
-//                      to global memory.
-//   producer (warp 9)  reads the records and issues TMA loads: one approximate tile per chunk
-//                      (KC chunk, mean-V chunk) and K_j / V_j ONLY for routed blocks.
-//   mma      (warps 10, 11) one thread each issues tcgen05.mma: warp 10 the score GEMMs S = Q K^T,
-//                      warp 11 the value GEMMs O += P V.  S goes to one of two TMEM score buffers,
-//                      so the scores of tile g+1 are computed while tile g is in softmax.
+//                      record (flat list of tile descriptors + per-column bias); nothing of the
+//                      proxy map goes to global memory.
+//   producer (warp 9, one lane) reads the records and issues TMA loads: one approximate tile per
+//                      chunk (KC chunk, mean-V chunk) and K_j / V_j ONLY for routed blocks.
+//   mma      (warps 10, 11) issue tcgen05.mma: warp 10 the score GEMMs S = Q K^T, warp 11 the value
+//                      GEMMs O += P V; each warp runs in lockstep and one elected lane issues.  S
+//                      goes to one of two TMEM score buffers, so the scores of tile g+1 are
+//                      computed while tile g is in softmax.
 //   softmax  (warps 0-3 and 4-7) two warpgroups; thread = query row; group h owns key columns
 //                      [64h, 64h+64) of EVERY tile and keeps its own running (m_h, l_h) and its own
 //                      accumulator O_h in TMEM (O_h += P_h V[64h:64h+64]); the two partial results
@@ -162,7 +163,7 @@ __device__ long long g_trace[kTraceTiles * kTraceEvents];
 #endif
 
 // ------------------------------------------------------------------------------------------------
-// Every consumer role (producer, the two MMA threads, both softmax warpgroups) walks the record
+// Every consumer role (producer, the two MMA warps, both softmax warpgroups) walks the record
 // ring with a cursor of its own and sees the same flat stream of descriptors.
 struct Cursor {
   uint32_t n_rec = 0;
@@ -785,7 +786,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     sm.abort_flag = 0;
-    // a record is released by the two producers, the two MMA threads and the 8 softmax warps
+    // a record is released by the producer's two cursors, the two MMA warps and the 8 softmax warps
     for (int r = 0; r < kRecords; ++r) { mbar_init(&sm.rec_full[r], 1); mbar_init(&sm.rec_empty[r], 12); }
     for (int s = 0; s < kKStages; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
