@@ -3,18 +3,22 @@ debug mask, and comparing the CUDA path with the CPU oracle under the acceptance
 
 * block mask identical to the oracle's except for blocks whose proxy score lies within 1e-3
   of the threshold (their number is reported);
-* output max-abs error <= 1e-2 and relative L2 error <= 5e-3 (bf16 I/O, fp32 accumulation),
-  judged against the oracle evaluated under the GPU's mask for tiles with an in-band flip.
-
-The absolute bound is stated for outputs of order one.  Three bf16 roundings sit on the path of
-every output element -- the value operand (V, or the pooled mean value of the approximate
-branch), the probability P fed to the tensor core, and the stored output -- each up to 2^-8
-relative, and they do not average out in a row whose attention mass sits on a single key or
-block.  For |reference| > 1 the bound is therefore applied as a relative one:
-|error| <= 1e-2 * max(1, |reference|).  Elements with |reference| <= 1 must meet 1e-2 as stated;
-the plain max-abs error and the max-abs error over |reference| <= 1 are both reported.
+* relative L2 error of the output <= 5e-3;
+* output max-abs error <= 1e-2 (bf16 I/O, fp32 accumulation) for every element whose oracle
+  value is below 2 in magnitude.  The stored output is a bf16 number, whose spacing (ulp) is
+  2^-7 = 7.8e-3 on [1, 2): the stated 1e-2 is 1.28 ulp there.  On [2, 4) the spacing is 2^-6,
+  so rounding the exact result to bf16 already costs up to 7.8e-3 and the same 1.28-ulp
+  allowance reads 2e-2 (4e-2 on [4, 8) and so on).  The bound is therefore
+  ``max(1e-2, 1.28 * ulp_bf16(oracle))`` per element, and three figures are reported:
+  the plain max-abs error, the max-abs error over |oracle| < 2 (this one must meet 1e-2 as
+  stated), and the max-abs error against the oracle value rounded to bf16 (which takes the
+  output rounding out and shows what the bf16 operands P, KC and mean V contribute);
+* outputs of a tile with an in-band mask flip are judged against the oracle evaluated under the
+  GPU's mask, and reported under both masks.
 """
 from __future__ import annotations
+
+from dataclasses import dataclass
 
 import numpy as np
 import torch
@@ -26,11 +30,53 @@ from paper_2607_24027_b200 import synth
 BAND = 1e-3
 MAX_ABS = 1e-2
 REL_L2 = 5e-3
+ULPS = MAX_ABS / 2.0 ** -7          # 1.28 bf16 ulps of [1, 2)
+
+
+def bf16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 numbers (8 significant bits) around x."""
+    ax = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(ax)) - 7)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """x rounded to the nearest bf16 value (ties to even), as float64."""
+    return synth.widen(synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32)), np.float64)
 
 
 def out_bound(ref: np.ndarray) -> np.ndarray:
-    """Elementwise bound on |gpu - oracle|: 1e-2 absolute, relative beyond |oracle| = 1."""
-    return MAX_ABS * np.maximum(1.0, np.abs(ref))
+    """Elementwise bound on |gpu - oracle|: 1e-2, or 1.28 bf16 ulps of the oracle value where that is more."""
+    return np.maximum(MAX_ABS, ULPS * bf16_ulp(ref))
+
+
+def error_stats(got: np.ndarray, ref: np.ndarray) -> dict:
+    """The three error figures of one comparison (plus relative L2); raises on a violation."""
+    assert np.isfinite(got).all(), "GPU output has non-finite values"
+    err = np.abs(got - ref)
+    lt2 = np.abs(ref) < 2.0
+    st = {
+        "max_abs": float(err.max()),
+        "max_abs_ref_lt_2": float(err[lt2].max()) if lt2.any() else 0.0,
+        "max_abs_vs_bf16_oracle": float(np.abs(got - bf16_round(ref)).max()),
+        "n_over_1e-2": int((err > MAX_ABS).sum()),
+        "rel_l2": float(np.linalg.norm(got - ref) / np.linalg.norm(ref)),
+        "max_abs_out": float(np.abs(ref).max()),
+    }
+    assert st["max_abs_ref_lt_2"] <= MAX_ABS, st
+    assert (err <= out_bound(ref)).all(), st
+    assert st["rel_l2"] <= REL_L2, st
+    return st
+
+
+def merge_stats(a: dict, b: dict) -> dict:
+    """Worst case of two stats dicts (sums for the counters)."""
+    if not a:
+        return dict(b)
+    out = {}
+    for key in set(a) | set(b):
+        x, y = a.get(key, 0), b.get(key, 0)
+        out[key] = x + y if key in ("in_band_flips", "in_band_blocks", "blocks", "n_over_1e-2", "tiles") else max(x, y)
+    return out
 
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
@@ -51,7 +97,7 @@ def unpack_mask(words: torch.Tensor, n_k: int) -> np.ndarray:
 
 
 def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, scale=0.0, want_mask=True,
-            tau_override=None, ws=None, estimator=0, forced=None, layout=0):
+            tau_override=None, ws=None, estimator=0, forced=None, layout=0, skip_pool=False):
     """Run the fused forward through the C ABI; returns (out, counts, mask or None, ws).
 
     layout = SOL_LAYOUT_BNHD: q, k, v (and the returned out) are [B, N, H, d].
@@ -68,6 +114,7 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
         mask_words = torch.zeros(B, H, ws.view.n_q_blocks, sb.mask_words(nk), dtype=torch.int32, device="cuda")
     sb.sol_attn_forward_ex(q, k, v, out, ws, block, block, threshold=beta, scale=scale, mode=mode, impl=impl,
                            mask_out=mask_words, tau_override=tau_override, estimator=estimator, layout=layout,
+                           skip_pool=skip_pool,
                            forced_blocks=(None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.uint8)).cuda()))
     torch.cuda.synchronize()
     sb.sol_attn_bind_workspace(ws)
@@ -77,49 +124,88 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
     return out, ws.counts.clone(), mask, ws
 
 
-def check_head(qh, kh, vh, out_h, mask_h, counts_h, block, beta, tiles=None, scale=None, mode="sol",
-               estimator="direct", forced=None):
-    """Compare one head of GPU results with the oracle.
+# ------------------------------------------------------------------------------- oracle side, per head
+@dataclass
+class HeadRouting:
+    """Everything of the oracle's pre-attention step that does not depend on beta."""
+    qbar: np.ndarray
+    kc: np.ndarray
+    vc: np.ndarray
+    s_hat: np.ndarray      # [Nq, Nk] proxy scores (Eq. 3)
 
-    qh, kh, vh: float64 [L, d] inputs; out_h: float64 [L, d] GPU output; mask_h: [Nq, Nk] bool GPU
-    mask (or None); counts_h: [Nq] GPU counts (or None); tiles: query blocks whose OUTPUT is
-    checked (None = all).  Returns a dict of error statistics; raises on a violation.
-    """
-    L, d = qh.shape
-    r = orc.routing(qh, kh, vh, block, block, beta, scale=scale, estimator=estimator, forced=forced)
-    nq = r.mask.shape[0]
-    stats = {"in_band_flips": 0, "blocks": int(r.mask.size)}
-    override = r.mask if forced is not None else None
+    def at(self, beta, estimator="direct", scale=None):
+        """(mu, sigma, tau, mask) of Eq. (4) for one beta."""
+        if estimator == "direct":
+            mu, sigma, tau = orc.threshold_direct(self.s_hat, beta)
+        else:
+            s = orc.default_scale(self.qbar.shape[1]) if scale is None else scale
+            mu, sigma, tau = orc.threshold_diagonal(self.qbar, self.kc, beta, s)
+        return mu, sigma, tau, orc.select_blocks(self.s_hat, tau)
+
+
+def head_routing(qh, kh, vh, block, scale=None) -> HeadRouting:
+    s = orc.default_scale(qh.shape[1]) if scale is None else scale
+    qbar, kc, vc, _ = orc.pool(qh, kh, vh, block, block)
+    return HeadRouting(qbar=qbar, kc=kc, vc=vc, s_hat=orc.proxy_scores(qbar, kc, s))
+
+
+def check_mask(mask_h, counts_h, s_hat, tau, ref_mask) -> dict:
+    """GPU mask / counts of one head against the oracle's: identical outside the 1e-3 band."""
+    band = np.abs(s_hat - tau[:, None]) < BAND
+    st = {"blocks": int(ref_mask.size), "in_band_blocks": int(band.sum()), "in_band_flips": 0}
     if mask_h is not None:
-        diff = mask_h != r.mask
-        band = np.abs(r.s_hat - r.tau[:, None]) < BAND
+        diff = mask_h != ref_mask
         assert not (diff & ~band).any(), f"{int((diff & ~band).sum())} mask mismatches outside the 1e-3 band"
-        stats["in_band_flips"] = int(diff.sum())
-        stats["in_band_blocks"] = int(band.sum())
-        if diff.any():
-            override = mask_h
+        st["in_band_flips"] = int(diff.sum())
         if counts_h is not None:
             assert np.array_equal(counts_h, mask_h.sum(axis=1)), "counts disagree with the GPU's own mask"
     elif counts_h is not None:
-        band = np.abs(r.s_hat - r.tau[:, None]) < BAND
-        assert (np.abs(counts_h - r.counts) <= band.sum(axis=1)).all(), "counts differ beyond in-band blocks"
-    tiles = list(range(nq)) if tiles is None else list(tiles)
-    o, _ = orc.sol_attn_streaming(qh, kh, vh, r.kc, r.vc, r.tau, block, block, chunk=16, scale=scale,
+        assert (np.abs(counts_h - ref_mask.sum(axis=1)) <= band.sum(axis=1)).all(), "counts differ beyond in-band blocks"
+    return st
+
+
+def check_output(qh, kh, vh, out_h, kc, vc, tau, block, tiles, override=None, scale=None, mode="sol") -> dict:
+    """GPU output rows of the query blocks `tiles` against Algorithm 1 run by the oracle."""
+    L = qh.shape[0]
+    o, _ = orc.sol_attn_streaming(qh, kh, vh, kc, vc, tau, block, block, chunk=16, scale=scale,
                                   q_tiles=tiles, mask_override=override, exact_only=(mode == "exact_only"))
     rows = np.concatenate([np.arange(i * block, min((i + 1) * block, L)) for i in tiles])
     ref, got = o[rows], out_h[rows]
     if mode == "exact_only":      # query blocks that route nothing have no defined output
         keep = np.isfinite(ref).all(axis=1)
         ref, got = ref[keep], got[keep]
-    assert np.isfinite(got).all(), "GPU output has non-finite values"
-    err = np.abs(got - ref)
-    bound = out_bound(ref)
-    small = np.abs(ref) <= 1.0
-    stats["max_abs"] = float(err.max())
-    stats["max_abs_ref_le_1"] = float(err[small].max()) if small.any() else 0.0
-    stats["worst_ratio_to_bound"] = float((err / bound).max())
-    stats["rel_l2"] = float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
-    stats["max_abs_out"] = float(np.abs(ref).max())
-    assert (err <= bound).all(), stats
-    assert stats["rel_l2"] <= REL_L2, stats
+    st = error_stats(got, ref)
+    st["tiles"] = len(tiles)
+    return st
+
+
+def check_head(qh, kh, vh, out_h, mask_h, counts_h, block, beta, tiles=None, scale=None, mode="sol",
+               estimator="direct", forced=None, routing=None):
+    """Compare one head of GPU results with the oracle.
+
+    qh, kh, vh: float64 [L, d] inputs; out_h: float64 [L, d] GPU output; mask_h: [Nq, Nk] bool GPU
+    mask (or None); counts_h: [Nq] GPU counts (or None); tiles: query blocks whose OUTPUT is
+    checked (None = all); routing: a HeadRouting computed earlier for this head (else made here).
+    Returns a dict of error statistics; raises on a violation.
+    """
+    r = routing if routing is not None else head_routing(qh, kh, vh, block, scale=scale)
+    _, _, tau, ref_mask = r.at(beta, estimator=estimator, scale=scale)
+    if forced is not None:
+        ref_mask = ref_mask | np.asarray(forced, dtype=bool)[None, :]
+    stats = check_mask(mask_h, counts_h, r.s_hat, tau, ref_mask)
+    override = ref_mask if forced is not None else None
+    flipped = []
+    if mask_h is not None and stats["in_band_flips"]:
+        override = mask_h
+        flipped = np.flatnonzero((mask_h != ref_mask).any(axis=1)).tolist()
+    nq = ref_mask.shape[0]
+    tiles = list(range(nq)) if tiles is None else sorted(set(tiles) | set(flipped[:16]))
+    stats.update(check_output(qh, kh, vh, out_h, r.kc, r.vc, tau, block, tiles, override=override, scale=scale,
+                              mode=mode))
+    if flipped:                   # the same tiles under the oracle's own mask: reported, not asserted
+        o, _ = orc.sol_attn_streaming(qh, kh, vh, r.kc, r.vc, tau, block, block, chunk=16, scale=scale,
+                                      q_tiles=flipped[:16], mask_override=ref_mask,
+                                      exact_only=(mode == "exact_only"))
+        rows = np.concatenate([np.arange(i * block, min((i + 1) * block, qh.shape[0])) for i in flipped[:16]])
+        stats["max_abs_flipped_tiles_under_oracle_mask"] = float(np.nanmax(np.abs(out_h[rows] - o[rows])))
     return stats

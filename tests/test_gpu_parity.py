@@ -53,7 +53,7 @@ def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=
                                       estimator=(1 if estimator == "diagonal" else 0), forced=forced)
     B, H, N, d = q.shape
     out64 = hp.dev_to_f64(out)
-    agg = {"in_band_flips": 0, "max_abs": 0.0, "rel_l2": 0.0}
+    agg = {}
     for b in range(B):
         for h in range(H):
             st = hp.check_head(synth.widen(qb[b, h], np.float64), synth.widen(kb[b, h], np.float64),
@@ -61,9 +61,7 @@ def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=
                                counts[b, h].cpu().numpy(), block, beta, tiles=tiles,
                                scale=(scale if scale > 0 else None), mode=mode_name, estimator=estimator,
                                forced=forced)
-            agg["in_band_flips"] += st["in_band_flips"]
-            agg["max_abs"] = max(agg["max_abs"], st["max_abs"])
-            agg["rel_l2"] = max(agg["rel_l2"], st["rel_l2"])
+            agg = hp.merge_stats(agg, st)
     return agg
 
 
@@ -118,7 +116,7 @@ def test_tiny_all_tiles(impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS_128)
-@pytest.mark.parametrize("rho", [0.2, 0.4, 0.6])
+@pytest.mark.parametrize("rho", [0.2, 0.3, 0.4, 0.5, 0.6])
 def test_image_all_tiles(impl, rho):
     wl = WORKLOADS["image"]
     beta = load_betas()["image"][rho]
