@@ -67,8 +67,8 @@ enum {
 
 /* which implementation of the fused kernel runs */
 enum {
-  SOL_IMPL_AUTO     = 0,  /* tcgen05 kernel when the shape allows it, else the mma.sync one    */
-  SOL_IMPL_TCGEN05  = 1,  /* TMA + tcgen05.mma + TMEM kernel (d = 128, block 128)              */
+  SOL_IMPL_AUTO     = 0,  /* the tcgen05 kernel                                                */
+  SOL_IMPL_TCGEN05  = 1,  /* TMA + tcgen05.mma + TMEM kernel (all supported shapes)            */
   SOL_IMPL_MMA_SYNC = 2   /* portable warp-level mma.sync kernel (all supported shapes)        */
 };
 
@@ -243,6 +243,15 @@ sol_status_t sol_attn_route_materialized(const float* qbar, const float* kc, int
 
 /* Number of kernels the library has launched since it was loaded (for launch accounting). */
 int64_t sol_attn_launch_count(void);
+
+/* Testing hook for the device-side failure path (the paper has no counterpart).  Every wait inside the
+ * tcgen05 kernel is bounded; this call sets, for all later launches of the process, the bound in SM
+ * clocks (wait_cycles <= 0 restores the default of about two seconds) and the index of one tile per CTA
+ * whose "value GEMM finished" signal is left out (withhold_tile < 0: none).  With a tile withheld the
+ * waits on that signal run out, every warp role drains, TMEM is released, the kernel returns and
+ * sol_attn_read_device_status() reports SOL_ERR_DEVICE_TIMEOUT; the outputs of that launch are invalid.
+ * Nothing faults, traps or spins without a bound.  Not for production use; not thread-safe. */
+void sol_attn_debug_set_wait(int64_t wait_cycles, int32_t withhold_tile);
 
 #ifdef __cplusplus
 }

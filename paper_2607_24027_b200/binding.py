@@ -36,7 +36,7 @@ EXPORTS = [
     "sol_attn_bind_workspace", "sol_attn_pool", "sol_attn_forward", "sol_attn_dense",
     "sol_attn_forward_ex", "sol_attn_forward_host", "sol_attn_read_device_status",
     "sol_attn_launch_count", "sol_attn_thresholds_static", "sol_attn_thresholds_static_max_floats",
-    "sol_attn_route_materialized", "sol_attn_thresholds",
+    "sol_attn_route_materialized", "sol_attn_thresholds", "sol_attn_debug_set_wait",
 ]
 
 
@@ -113,6 +113,8 @@ def lib() -> ctypes.CDLL:
     L.sol_attn_route_materialized.argtypes = [ctypes.c_void_p] * 2 + [ctypes.c_int] * 5 + [ctypes.c_float, ctypes.c_int,
                                                                                            ctypes.c_float] + \
                                              [ctypes.c_void_p] * 5
+    L.sol_attn_debug_set_wait.restype = None
+    L.sol_attn_debug_set_wait.argtypes = [ctypes.c_int64, ctypes.c_int32]
     _lib = L
     return L
 
@@ -305,6 +307,12 @@ def sol_attn_read_device_status(stream=None) -> int:
 
 def sol_attn_launch_count() -> int:
     return int(lib().sol_attn_launch_count())
+
+
+def sol_attn_debug_set_wait(wait_cycles: int = 0, withhold_tile: int = -1):
+    """Testing hook: bound of the kernel's device-side waits (SM clocks, <= 0: default) and the tile per CTA
+    whose completion signal is withheld (< 0: none)."""
+    lib().sol_attn_debug_set_wait(int(wait_cycles), int(withhold_tile))
 
 
 def mask_words(n_k_blocks: int) -> int:

@@ -332,4 +332,8 @@ sol_status_t sol_attn_read_device_status(sol_stream_t stream) {
 
 int64_t sol_attn_launch_count(void) { return g_launches.load(); }
 
+void sol_attn_debug_set_wait(int64_t wait_cycles, int32_t withhold_tile) {
+  sol::fwd_sm100_set_wait(static_cast<long long>(wait_cycles), withhold_tile);
+}
+
 }  // extern "C"

@@ -116,8 +116,11 @@ cudaError_t launch_fwd_mma_sync(const Problem& p, const __nv_bfloat16* q, const 
                                 const float* tau, int32_t* counts, uint32_t* mask_out,
                                 cudaStream_t stream, int* n_launches);
 
-// Fused forward, TMA + tcgen05 + TMEM implementation (d = 128, block 128).
+// Fused forward, TMA + tcgen05 + TMEM implementation (d in {64, 128}, block_q = block_k in {64, 128}).
 bool fwd_sm100_supports(const Problem& p);
+// Test hook: SM clocks after which the kernel's bounded waits give up (<= 0: the default) and the tile
+// whose P V completion signal each CTA leaves out (< 0: none); applies to the following launches.
+void fwd_sm100_set_wait(long long wait_cycles, int withhold_tile);
 cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, __nv_bfloat16* out, const WsPtrs& ws,
                              const float* tau, int32_t* counts, uint32_t* mask_out,

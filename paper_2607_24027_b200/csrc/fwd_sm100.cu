@@ -1,10 +1,11 @@
 // Sol-Attn fused forward (Algorithm 1) for sm_100a: TMA + tcgen05.mma + TMEM.
 //
-// Persistent kernel, one CTA of 384 threads per SM, d = 128, block_q = block_k = 128.  A CTA owns
-// one query block at a time and is split into warp roles that talk through mbarriers:
+// Persistent kernel, one CTA of 384 threads per SM, compiled for d in {64, 128} and
+// block_q = block_k in {64, 128}.  A CTA owns one query block at a time and is split into warp
+// roles that talk through mbarriers:
 //
 //   router   (warp 8)  pulls (head, query block) work items from a global counter and walks the
-//                      pooled keys in chunks of 128 blocks.  For every block it evaluates the
+//                      pooled keys in chunks of `block` blocks.  For every block it evaluates the
 //                      proxy s_ij = scale * Qbar_i . KC_j (Eq. 3) in fp32 and compares it with
 //                      tau_i (Eq. 4).  The decision only ever lives in a small shared-memory
 //                      record (flat list of tile descriptors + per-column bias); nothing of the
@@ -16,17 +17,21 @@
 //                      goes to one of two TMEM score buffers, so the scores of tile g+1 are
 //                      computed while tile g is in softmax.
 //   softmax  (warps 0-3 and 4-7) two warpgroups; thread = query row; group h owns key columns
-//                      [64h, 64h+64) of EVERY tile and keeps its own running (m_h, l_h) and its own
-//                      accumulator O_h in TMEM (O_h += P_h V[64h:64h+64]); the two partial results
-//                      are merged when the query block is finished.  Both branches of the method
+//                      [block/2 * h, block/2 * (h+1)) of EVERY tile and keeps its own running
+//                      (m_h, l_h) and its own accumulator O_h in TMEM; the two partial results are
+//                      merged when the query block is finished.  Both branches of the method
 //                      update the same state: an approximate tile is an ordinary tile whose
 //                      columns carry the bias log2(n_j) (Eqs. 9-10: multiplicity n_j in the
 //                      denominator, mean value times n_j in the numerator) or -inf for routed /
 //                      padded columns.  O_h is rescaled lazily, only when the running maximum
 //                      grows by more than 2^8.
 //
-// TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512); P_h (bf16) of a tile
-// overwrites the first 32 columns of group h's half of that tile's S buffer.
+// The query tile of the MMAs always has 128 rows (the M of a one-CTA tcgen05.mma at full rate);
+// with 64-token blocks its upper 64 rows belong to the next query block, take part in the
+// arithmetic and are never stored.
+//
+// TMEM (512 columns): S0 [0, block)  S1 [block, 2 block)  O0 [256, 256 + d)  O1 [256 + d, 256 + 2 d);
+// P_h (bf16) of a tile overwrites the start of group h's half of that tile's S buffer.
 //
 // Every mbarrier wait is bounded: when one expires the CTA records SOL_ERR_DEVICE_TIMEOUT in the
 // workspace status word, all roles drain, TMEM is released and the kernel returns.
@@ -39,15 +44,10 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128;
-constexpr int kBlk = 128;
-constexpr int kHalf = 64;                        // key columns per softmax warpgroup
+constexpr int kRowsQ = 128;                      // rows of the query tile fed to the tensor core
 constexpr int kThreads = 384;
-constexpr int kTileBytes = kBlk * kD * 2;        // 32 KB: one K-like or V-like tile
-constexpr int kHalfBytes = kTileBytes / 2;       // 16 KB: 64 channels x 128 rows (one TMA box)
 constexpr int kKStages = 2;                      // ring of K tiles
 constexpr int kVStages = 2;                      // ring of V tiles (its own ring: the score GEMMs run ahead of P V)
-constexpr int kStages = kKStages + kVStages;
 constexpr int kGroup = 32;                       // pooled keys scored per router step (one per lane)
 constexpr int kRecords = 4;                      // ring of routing records
 constexpr int kWarpRouter = 8, kWarpProducer = 9, kWarpQK = 10;   // warp 11 issues P V
@@ -55,7 +55,22 @@ constexpr int kTmemCols = 512;
 constexpr int kTmemS = 0, kTmemO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units
 
-// The router turns every chunk of 128 key blocks into a record: a flat list of tile descriptors
+// Compile-time shape of one kernel instance.
+template <int D, int BLK>
+struct Cfg {
+  static constexpr int kD = D;                     // head dimension
+  static constexpr int kBlk = BLK;                 // block_q = block_k = key columns of a tile
+  static constexpr int kHalf = BLK / 2;            // key columns per softmax warpgroup
+  static constexpr int kBoxes = D / 64;            // 64-channel TMA boxes per tile row
+  static constexpr int kQBytes = kRowsQ * D * 2;   // the query tile
+  static constexpr int kTileBytes = BLK * D * 2;   // one K-like or V-like tile
+  static constexpr int kQBoxBytes = kRowsQ * 128;  // one box of the query tile (64 channels x 128 rows)
+  static constexpr int kBoxBytes = BLK * 128;      // one box of a K-like / V-like tile
+  static_assert(D == 64 || D == 128, "head dimension");
+  static_assert(BLK == 64 || BLK == 128, "block size");
+};
+
+// The router turns every chunk of `block` key blocks into a record: a flat list of tile descriptors
 // that the other roles only have to read.  A descriptor is (row coordinate << 5) | flags; the
 // coordinate is the first key row of an exact tile or the first pooled row of an approximate one.
 constexpr uint32_t kTileApprox = 1;      // approximate-branch tile (pooled keys / mean values)
@@ -64,26 +79,29 @@ constexpr uint32_t kTileEnd = 4;         // not a tile: the work item ends here
 constexpr uint32_t kTileEmptyItem = 8;   // on an end entry: the item had no tile at all
 constexpr uint32_t kDescStop = 0xffffffffu, kDescAbort = 0xfffffffeu, kDescNone = 0xfffffffdu;
 
+template <class C>
 struct alignas(16) Record {
-  float bias[kBlk];             // approximate-tile column bias: log2(n_j) / (scale * log2 e), or -inf
+  float bias[C::kBlk];          // approximate-tile column bias: log2(n_j) / (scale * log2 e), or -inf
   int32_t work;                 // bh * Nq + i, or -1: no more work
   int32_t b, h;                 // batch and head of the work item
   int32_t q_row;                // first query row of the work item
   int16_t first, end;           // descriptors [first, end) are valid (slot 0 is kept for the approximate tile)
-  uint32_t desc[kBlk + 2];
+  uint32_t desc[C::kBlk + 2];
 };
 
+template <class C>
 struct Shared {
-  float kc_stage[2][kGroup * kD];   // router: fp32 pooled keys of the group being scored / the next one
-  float qbar_s[kD];                 // router: pooled query of the current work item
-  Record rec[kRecords];
-  float2 ml[2][kBlk];           // (m_h, l_h) exchange between the softmax warpgroups
+  float kc_stage[2][kGroup * C::kD];   // router: fp32 pooled keys of the group being scored / the next one
+  float qbar_s[C::kD];                 // router: pooled query of the current work item
+  Record<C> rec[kRecords];
+  float2 ml[2][kRowsQ];         // (m_h, l_h) exchange between the softmax warpgroups
   uint64_t rec_full[kRecords], rec_empty[kRecords];
   uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
   uint64_t q_full, q_empty;
   uint64_t s_full[2], p_full[2][2], pv_done[2];   // indexed by score buffer (and warpgroup)
   uint64_t x_full, x_done;      // rendezvous of the two softmax warpgroups at the end of a work item
   uint64_t kc_full[2];          // router staging buffers filled
+  uint64_t mma_drain[2];        // abort path only: all MMAs issued by a role have retired
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -101,82 +119,60 @@ struct Params {
   const uint8_t* forced;        // [Nk] or null: key blocks always routed to the exact branch
   Strides st;                   // layout of q, k, v, out
   int rows_inner;               // coordinate order of the q/k/v tensor maps: (c, row, h, b) or (c, h, row, b)
+  long long wait_limit;         // SM clocks after which a bounded wait gives up
+  int withhold_tile;            // test hook: >= 0: the P V role leaves out the completion signal of this tile
 };
 
-__device__ __forceinline__ void flag_abort(Shared& sm, const Params& p, int where) {
+template <class S>
+__device__ __forceinline__ void flag_abort(S& sm, const Params& p, int where) {
   sm.abort_flag = 1;
   atomicExch(p.status + kStatusDevice, (int)SOL_ERR_DEVICE_TIMEOUT);
   atomicCAS(p.status + kStatusDetail, 0, where);     // keep the first place that gave up
 }
 
-// Optional per-role cycle accounting (build with -DSOL_PROFILE): how long each role spends in
-// each kind of wait.  Slot meaning is listed next to every use; read back with
-// sol_attn_debug_profile().
-#ifdef SOL_PROFILE
-constexpr int kProfCtas = 512, kProfRoles = 4, kProfSlots = 12;
-__device__ long long g_prof[kProfCtas * kProfRoles * kProfSlots];
-struct Prof {
-  long long v[kProfSlots];
-  long long t0;
-  __device__ Prof() {
-    for (int i = 0; i < kProfSlots; ++i) v[i] = 0;
-    t0 = clock64();
-  }
-  __device__ void flush(int role) {
-    v[kProfSlots - 1] = clock64() - t0;
-    if (blockIdx.x < kProfCtas)
-      for (int i = 0; i < kProfSlots; ++i) g_prof[(blockIdx.x * kProfRoles + role) * kProfSlots + i] = v[i];
-  }
-};
-__device__ __forceinline__ bool prof_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long& acc) {
-  const long long t = clock64();
-  const bool ok = mbar_wait(bar, parity, abort_flag);
-  acc += clock64() - t;
-  return ok;
-}
-#define WAIT(bar, parity, slot) prof_wait((bar), (parity), &sm.abort_flag, prof.v[slot])
-#define PROF_DECL Prof prof;
-#define PROF_COUNT(slot) (++prof.v[slot])
-#define PROF_FLUSH(role) prof.flush(role)
-#define PROF_ACC(slot) (&prof.v[slot])
-// timeline of a few tiles of CTA 0: [tile][event] = clock64()
-#ifndef SOL_TRACE_FIRST
-#define SOL_TRACE_FIRST 40
+}  // namespace
+}  // namespace sol
+
+// Every role has `sm` and `wait_limit` in scope; WAIT is a bounded wait on one of its barriers.
+#if defined(SOL_PROFILE) || defined(SOL_ITEMTRACE)
+#include "fwd_sm100_prof.cuh"
 #endif
-constexpr int kTraceFirst = SOL_TRACE_FIRST, kTraceTiles = 16, kTraceEvents = 80;
-__device__ long long g_trace[kTraceTiles * kTraceEvents];
-#define TRACE(tile, evt) do { if (blockIdx.x == 0 && (tile) >= kTraceFirst && (tile) < kTraceFirst + kTraceTiles) g_trace[((tile) - kTraceFirst) * kTraceEvents + (evt)] = clock64(); } while (0)
-// per-warp phases of the softmax role: events 32 + 6 * warp + k
-#define WTRACE(k) do { if (lane == 0) TRACE(g, 32 + (4 * h + warp_in_group) * 6 + (k)); } while (0)
-#define PROF_T0 const long long prof_t0 = clock64();
-#define PROF_ADD(slot) prof.v[slot] += clock64() - prof_t0;
+#ifdef SOL_PROFILE
+#define WAIT(bar, parity, slot) SOL_WAIT(bar, parity, slot)
 #else
-#define WAIT(bar, parity, slot) mbar_wait((bar), (parity), &sm.abort_flag)
+#define WAIT(bar, parity, slot) mbar_wait((bar), (parity), &sm.abort_flag, wait_limit)
 #define PROF_DECL
 #define PROF_COUNT(slot)
 #define PROF_FLUSH(role)
 #define PROF_ACC(slot) nullptr
-#define TRACE(tile, evt)
-#define WTRACE(k)
 #define PROF_T0
 #define PROF_ADD(slot)
 #endif
+#ifndef SOL_ITEMTRACE
+#define ITRACE(item, slot)
+#define ITRACE_VAL(item, slot, val)
+#define CTATRACE(slot, val)
+#endif
+
+namespace sol {
+namespace {
 
 // ------------------------------------------------------------------------------------------------
 // Every consumer role (producer, the two MMA warps, both softmax warpgroups) walks the record
 // ring with a cursor of its own and sees the same flat stream of descriptors.
+template <class C>
 struct Cursor {
   uint32_t n_rec = 0;
   int e = 0, end = 0;
-  const Record* rec = nullptr;   // the open record (valid until the next call)
+  const Record<C>* rec = nullptr;   // the open record (valid until the next call)
 };
 
 // `release` is called when the cursor is done with a record (arrives on rec_empty as appropriate
 // for the role).  Returns kDescStop at the end of the stream, kDescAbort when a bounded wait
 // expired and, with block = false, kDescNone when the next record has not been written yet.
-template <class Release>
-__device__ __forceinline__ uint32_t next_desc(Shared& sm, Cursor& c, long long* wait_acc, Release release,
-                                              bool block = true) {
+template <class C, class Release>
+__device__ __forceinline__ uint32_t next_desc(Shared<C>& sm, Cursor<C>& c, long long wait_limit, long long* wait_acc,
+                                              Release release, bool block = true) {
   for (;;) {
     if (c.e < c.end) return c.rec->desc[c.e++];
     if (c.rec) {
@@ -189,7 +185,7 @@ __device__ __forceinline__ uint32_t next_desc(Shared& sm, Cursor& c, long long* 
 #ifdef SOL_PROFILE
     const long long t = clock64();
 #endif
-    const bool ok = mbar_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1, &sm.abort_flag);
+    const bool ok = mbar_wait(&sm.rec_full[r], (c.n_rec / kRecords) & 1, &sm.abort_flag, wait_limit);
 #ifdef SOL_PROFILE
     if (wait_acc) *wait_acc += clock64() - t;
 #endif
@@ -203,33 +199,40 @@ __device__ __forceinline__ uint32_t next_desc(Shared& sm, Cursor& c, long long* 
 
 // ------------------------------------------------------------------------------------------------
 // router: one warp
-__device__ void router_role(Shared& sm, const Params& p, int lane) {
+template <class C>
+__device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
+  constexpr int kD = C::kD, kBlk = C::kBlk, kPieces = C::kD / 4;   // 16-byte pieces per pooled key
   const unsigned full = 0xffffffffu;
+  const long long wait_limit = p.wait_limit;
   uint32_t n_rec = 0, n_copy = 0, n_use = 0;   // records written; staging copies issued / consumed
+  uint32_t n_item = 0;
   const int n_chunks = ceil_div(p.Nk, kBlk);
   const int mask_words = ceil_div(p.Nk, 32);
   const float inv_sl2 = 1.f / (p.scale * 1.4426950408889634f);   // biases are stored in raw-score units
   bool alive = true;
   PROF_DECL
+  if (lane == 0) CTATRACE(0, prof::gtimer());
   while (alive) {
     int w = 0;
     if (lane == 0) w = atomicAdd(p.status + kStatusTileCounter, 1);
     w = __shfl_sync(full, w, 0);
     if (w >= p.total_work) break;
+    if (lane == 0) ITRACE(n_item, 0);
     const int bh = w / p.Nq, i = w - bh * p.Nq;
     // the pooled query of this work item goes to shared memory (one 16-byte piece per lane)
     float tau_i = 0.f;
     if (p.mode != SOL_MODE_DENSE) {
       __syncwarp();
-      reinterpret_cast<float4*>(sm.qbar_s)[lane] =
-          __ldg(reinterpret_cast<const float4*>(p.qbar + ((size_t)bh * p.Nq + i) * kD) + lane);
+      if (lane < kPieces)
+        reinterpret_cast<float4*>(sm.qbar_s)[lane] =
+            __ldg(reinterpret_cast<const float4*>(p.qbar + ((size_t)bh * p.Nq + i) * kD) + lane);
       tau_i = p.tau[(size_t)bh * p.Nq + i];
       __syncwarp();
     }
     const float* kc_head = p.kc + (size_t)bh * p.Nk * kD;
     int count = 0;
     bool item_has_tiles = false;
-    // Bulk-copy one group of 32 pooled keys (16 KB, contiguous in memory) into a staging buffer;
+    // Bulk-copy one group of 32 pooled keys (contiguous in memory) into a staging buffer;
     // the copy of group n+1 is in flight while group n is scored.
     auto stage_group = [&](int jb) {
       if (p.mode == SOL_MODE_DENSE || jb >= p.Nk) return;
@@ -245,7 +248,7 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
     };
     stage_group(0);
     for (int t = 0; t < n_chunks; ++t) {
-      Record& rec = sm.rec[n_rec % kRecords];
+      Record<C>& rec = sm.rec[n_rec % kRecords];
       if (!WAIT(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, 0)) {   // prof 0: record ring full
         if (lane == 0) flag_abort(sm, p, 100);
         alive = false;
@@ -263,8 +266,8 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
           sel = j < p.Nk;
         } else {
           // lane l scores pooled key jbase + l against the staged rows.  Lane l starts at 16-byte
-          // piece l of its row and of the query and walks round, so that the 32 lanes hit 32
-          // different shared-memory bank groups although the rows are 512 bytes apart.
+          // piece l of its row and of the query and walks round, so that the lanes spread over the
+          // shared-memory bank groups although the rows are a multiple of 128 bytes apart.
           float dot = 0.f;
           if (jbase < p.Nk) {
             const uint32_t buf = n_use & 1;
@@ -279,8 +282,8 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
             const float4* qv = reinterpret_cast<const float4*>(sm.qbar_s);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < kD / 4; ++c) {
-              const int piece = (c + lane) & (kD / 4 - 1);
+            for (int c = 0; c < kPieces; ++c) {
+              const int piece = (c + lane) & (kPieces - 1);
               const float4 kk = row[piece];
               const float4 qq = qv[piece];
               a0 = fmaf(qq.x, kk.x, a0);
@@ -301,11 +304,12 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
         n_sel += __popc(m);
         if (p.mask_out && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
       }
+      if (!alive) break;
       any_unselected = __any_sync(full, any_unselected);
       count += n_sel;
       const bool has_approx = p.mode == SOL_MODE_SOL && any_unselected;
       const int first = has_approx ? 0 : 1;
-      int end = 1 + n_sel;                   // n_sel <= 128
+      int end = 1 + n_sel;                   // n_sel <= block
       __syncwarp();
       if (lane == 0) {
         rec.work = w;
@@ -321,14 +325,23 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
       item_has_tiles |= end > first;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.rec_full[n_rec % kRecords]);
+      if (lane == 0 && t == 0) ITRACE(n_item, 1);
+      if (lane == 0 && t == n_chunks - 1) ITRACE(n_item, 2);
       ++n_rec;
     }
     if (alive && lane == 0 && p.counts) p.counts[w] = count;
+    ++n_item;
   }
+  if (lane == 0) { CTATRACE(1, prof::gtimer()); CTATRACE(2, (long long)n_item); }
   PROF_FLUSH(0);
+  if (!alive) {
+    // let a staging copy that is still in flight land before the CTA's shared memory goes away
+    int never = 0;                                   // this drain must not be cut short by the abort flag
+    for (; n_use != n_copy; ++n_use) mbar_wait(&sm.kc_full[n_use & 1], (n_use >> 1) & 1, &never, wait_limit);
+  }
   // end-of-stream record
   if (alive) {
-    if (mbar_wait(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, &sm.abort_flag)) {
+    if (mbar_wait(&sm.rec_empty[n_rec % kRecords], ((n_rec / kRecords) & 1) ^ 1, &sm.abort_flag, wait_limit)) {
       if (lane == 0) {
         sm.rec[n_rec % kRecords].work = -1;
         mbar_arrive(&sm.rec_full[n_rec % kRecords]);
@@ -344,21 +357,25 @@ __device__ void router_role(Shared& sm, const Params& p, int lane) {
 // ahead of the V loads: that is the order in which the slots come free (a K slot when its score
 // GEMM retires, a V slot a softmax pass and a P V later), so an in-order thread seldom waits for a
 // slot while another load could go.
-__device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV,
+template <class C>
+__device__ void producer_role(Shared<C>& sm, const Params& p, unsigned char* sQ, unsigned char* sKV,
                               const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vm) {
   constexpr int kLead = 2;
+  constexpr int kTileBytes = C::kTileBytes;
+  const long long wait_limit = p.wait_limit;
   uint32_t n_k = 0, n_v = 0, n_item = 0;
-  Cursor cur_k, cur_v;
+  Cursor<C> cur_k, cur_v;
   PROF_DECL
-  // pooled = true: KC / mean-V operands, dense [B*H][Nk][d]; else q, k, v in the caller's layout
-  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, const Record* rec,
-                       bool pooled) {
-    mbar_arrive_expect_tx(full, kTileBytes);
+  // pooled = true: KC / mean-V operands, dense [B*H][Nk][d]; else q, k, v in the caller's layout.
+  // A tile is C::kBoxes boxes of 64 channels, each `box_bytes` long in shared memory.
+  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, const Record<C>* rec,
+                       bool pooled, int bytes, int box_bytes) {
+    mbar_arrive_expect_tx(full, bytes);
     const bool rows_inner = pooled || p.rows_inner;
     const int c1 = rows_inner ? row : rec->h, c2 = rows_inner ? rec->h : row;
-    tma_load_4d(dst, tm, full, 0, c1, c2, rec->b);
-    tma_load_4d(dst + kHalfBytes, tm, full, 64, c1, c2, rec->b);
+#pragma unroll
+    for (int c = 0; c < C::kBoxes; ++c) tma_load_4d(dst + c * box_bytes, tm, full, 64 * c, c1, c2, rec->b);
   };
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
   bool k_end = false, have_k = false, ok = true;
@@ -369,7 +386,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
       if (!have_k) {
         // never sleep on the router while a V load is owed: the router may itself be waiting for
         // the V cursor to hand a record back
-        dk = next_desc(sm, cur_k, PROF_ACC(0), release, n_k == n_v);            // prof 0: no record yet
+        dk = next_desc(sm, cur_k, wait_limit, PROF_ACC(0), release, n_k == n_v);      // prof 0: no record yet
         if (dk == kDescNone) break;
         if (dk == kDescAbort) { ok = false; break; }
         if (dk == kDescStop) { k_end = true; break; }
@@ -382,7 +399,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
         const uint32_t par = (n_item & 1) ^ 1;
         if (n_k != n_v && !mbar_try_wait(&sm.q_empty, par)) break;
         if (!WAIT(&sm.q_empty, par, 2)) { ok = false; break; }                  // prof 2: Q slot busy
-        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, cur_k.rec, false);
+        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, cur_k.rec, false, C::kQBytes, C::kQBoxBytes);
         ++n_item;
         dk &= ~kTileFirst;
       }
@@ -392,10 +409,9 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
       {
         PROF_T0
         load_tile((dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes, (int)(dk >> 5),
-                  cur_k.rec, (dk & kTileApprox) != 0);
+                  cur_k.rec, (dk & kTileApprox) != 0, kTileBytes, C::kBoxBytes);
         PROF_ADD(4)                                                                    // prof 4: issuing K copies
       }
-      TRACE(n_k, 12);
       ++n_k;
     }
     if (!ok) break;
@@ -408,7 +424,7 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     {
       PROF_T0
       do {
-        dv = next_desc(sm, cur_v, nullptr, release);
+        dv = next_desc(sm, cur_v, wait_limit, nullptr, release);
       } while (dv < kDescNone && (dv & kTileEnd));
       PROF_ADD(6)                                                                      // prof 6: V cursor
     }
@@ -418,16 +434,15 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
     {
       PROF_T0
       load_tile((dv & kTileApprox) ? tm_vm : tm_v, &sm.v_full[s], sKV + (size_t)(kKStages + s) * kTileBytes,
-                (int)(dv >> 5), cur_v.rec, (dv & kTileApprox) != 0);
+                (int)(dv >> 5), cur_v.rec, (dv & kTileApprox) != 0, kTileBytes, C::kBoxBytes);
       PROF_ADD(5)                                                                      // prof 5: issuing V copies
     }
-    TRACE(n_v, 13);
     ++n_v;
   }
   if (ok) {
     // the V cursor still has to hand back the records that hold no further tile
     for (;;) {
-      const uint32_t dv = next_desc(sm, cur_v, nullptr, release);
+      const uint32_t dv = next_desc(sm, cur_v, wait_limit, nullptr, release);
       if (dv >= kDescNone) break;
     }
   } else {
@@ -437,13 +452,14 @@ __device__ void producer_role(Shared& sm, const Params& p, unsigned char* sQ, un
   if (sm.abort_flag) {
     // let copies that are still in flight land before the CTA's shared memory goes away
     int never = 0;                                   // this drain must not be cut short by the abort flag
+    if (n_item > 0) mbar_wait(&sm.q_full, (n_item - 1) & 1, &never, wait_limit);
     for (uint32_t back = 0; back < kKStages && back < n_k; ++back) {
       const uint32_t n = n_k - 1 - back;
-      mbar_wait(&sm.k_full[n % kKStages], (n / kKStages) & 1, &never);
+      mbar_wait(&sm.k_full[n % kKStages], (n / kKStages) & 1, &never, wait_limit);
     }
     for (uint32_t back = 0; back < kVStages && back < n_v; ++back) {
       const uint32_t n = n_v - 1 - back;
-      mbar_wait(&sm.v_full[n % kVStages], (n / kVStages) & 1, &never);
+      mbar_wait(&sm.v_full[n % kVStages], (n / kVStages) & 1, &never, wait_limit);
     }
   }
 }
@@ -460,14 +476,26 @@ __device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo) {
   return ((uint64_t)hi << 32) | lo;
 }
 
+// Abort path of an MMA-issuing role: TMEM must not be released while MMAs are still writing to it, so
+// the role asks for a completion signal behind everything it has issued and waits for it (bounded).
+template <class C>
+__device__ __forceinline__ void drain_mmas(Shared<C>& sm, uint64_t* bar, bool leader, long long wait_limit) {
+  if (leader) mma_commit(bar);
+  int never = 0;
+  mbar_wait(bar, 0, &never, wait_limit);
+}
+
 // S_b = Q K^T (warp 10)
-__device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsigned char* sKV, uint32_t tmem) {
-  const uint32_t idesc_qk = make_idesc_bf16(kBlk, kBlk, false, false);
+template <class C>
+__device__ void mma_qk_role(Shared<C>& sm, const Params& p, unsigned char* sQ, unsigned char* sKV, uint32_t tmem) {
+  constexpr int kD = C::kD, kBlk = C::kBlk, kTileBytes = C::kTileBytes;
+  const long long wait_limit = p.wait_limit;
+  const uint32_t idesc_qk = make_idesc_bf16(kRowsQ, kBlk, false, false);
   const uint32_t q_lo = (smem_addr(sQ) >> 4) | (1u << 16);
   const uint32_t kv_lo = (smem_addr(sKV) >> 4) | (1u << 16);
   uint32_t n_item = 0, g = 0;
   uint32_t slot = 0, slot_parity = 0;          // ring position of K(g)
-  Cursor cur;
+  Cursor<C> cur;
   PROF_DECL
   // The whole warp runs this role in lockstep and one elected lane issues: with warp-uniform control
   // flow and operands the compiler keeps descriptors and addresses in uniform registers, where the
@@ -476,36 +504,36 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
   auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
+    const uint32_t dsc = next_desc(sm, cur, wait_limit, PROF_ACC(0), release);        // prof 0: no record yet
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) {                         // every MMA that reads Q_i has been issued
       if (!(dsc & kTileEmptyItem) && leader) mma_commit(&sm.q_empty);
       continue;
     }
-    if (dsc & kTileFirst) {
+    const bool it_first = (dsc & kTileFirst) != 0;
+    if (it_first) {
+      if (leader) ITRACE(n_item, 3);
       if (!WAIT(&sm.q_full, n_item & 1, 1)) { ok = false; break; }                    // prof 1: Q not loaded
       ++n_item;
     }
     const uint32_t b = g & 1;
-    TRACE(g, 24);
     if (!WAIT(&sm.k_full[slot], slot_parity, 2)) { ok = false; break; }               // prof 2: K not loaded
-    TRACE(g, 14);
     if (g >= 2) {
       // P overwrites S: the P V of tile g-2 must have read P out of this buffer
       if (!WAIT(&sm.pv_done[b], ((g - 2) >> 1) & 1, 3)) { ok = false; break; }        // prof 3: score buffer busy
     }
-    TRACE(g, 25);
     tc_fence_after();
-    TRACE(g, 0);
     {
       PROF_T0
       const uint32_t k_lo = kv_lo + slot * (kTileBytes >> 4);
       const uint32_t d_tmem = tmem + kTmemS + b * kBlk;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
-        const uint32_t off = ((ks / 4) * kHalfBytes + (ks % 4) * 32) >> 4;
-        const uint64_t da = desc_from_lo(q_lo + off), db = desc_from_lo(k_lo + off);
+        // K-step ks: 16 channels = 32 bytes inside box ks / 4
+        const uint32_t off_q = ((ks / 4) * C::kQBoxBytes + (ks % 4) * 32) >> 4;
+        const uint32_t off_k = ((ks / 4) * C::kBoxBytes + (ks % 4) * 32) >> 4;
+        const uint64_t da = desc_from_lo(q_lo + off_q), db = desc_from_lo(k_lo + off_k);
         if (leader) mma_ss(d_tmem, da, db, idesc_qk, ks > 0);
       }
       if (leader) {
@@ -513,39 +541,44 @@ __device__ void mma_qk_role(Shared& sm, const Params& p, unsigned char* sQ, unsi
         mma_commit(&sm.s_full[b]);
       }
       PROF_ADD(6)                                                                      // prof 6: issuing Q K^T
+      if (it_first && leader) ITRACE(n_item - 1, 4);
     }
-    TRACE(g, 1);
     ++g;
     if (++slot == kKStages) { slot = 0; slot_parity ^= 1; }
   }
   if (!ok && leader) flag_abort(sm, p, 300);
+  __syncwarp();
+  if (sm.abort_flag) drain_mmas(sm, &sm.mma_drain[0], leader, wait_limit);
   if (leader) PROF_FLUSH(2);
 }
 
-// O_h (+)= P_h V[64h : 64h+64], h = 0, 1 (warp 11)
-__device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uint32_t tmem) {
-  const uint32_t idesc_pv = make_idesc_bf16(kBlk, kD, false, true);
-  const uint32_t kv_lo = (smem_addr(sKV + kKStages * kTileBytes) >> 4) | ((uint32_t)(kHalfBytes >> 4) << 16);
+// O_h (+)= P_h V[half h of the tile's keys], h = 0, 1 (warp 11)
+template <class C>
+__device__ void mma_pv_role(Shared<C>& sm, const Params& p, unsigned char* sKV, uint32_t tmem) {
+  constexpr int kD = C::kD, kBlk = C::kBlk, kHalf = C::kHalf, kTileBytes = C::kTileBytes;
+  const long long wait_limit = p.wait_limit;
+  const uint32_t idesc_pv = make_idesc_bf16(kRowsQ, kD, false, true);
+  // V is the MN-major operand: its 64-channel boxes are C::kBoxBytes apart (leading offset), groups of
+  // 8 key rows 1024 bytes apart; a K-step of 16 keys advances the start by 2048 bytes.
+  const uint32_t kv_lo = (smem_addr(sKV + kKStages * kTileBytes) >> 4) | ((uint32_t)(C::kBoxBytes >> 4) << 16);
   uint32_t g = 0;
   uint32_t slot = 0, slot_parity = 0;          // ring position of V(g)
-  Cursor cur;
+  Cursor<C> cur;
   const bool leader = elect_one();             // warp-uniform role, one issuing lane (see mma_qk_role)
   auto release = [&](uint32_t r) { if (leader) mbar_arrive(&sm.rec_empty[r]); };
   bool ok = true;
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, nullptr, release);
+    const uint32_t dsc = next_desc(sm, cur, wait_limit, nullptr, release);
     if (dsc == kDescAbort) { ok = false; break; }
     if (dsc == kDescStop) break;
     if (dsc & kTileEnd) continue;
     const uint32_t b = g & 1;
-    if (!mbar_wait(&sm.v_full[slot], slot_parity, &sm.abort_flag)) { ok = false; break; }
-    TRACE(g, 2);
+    if (!mbar_wait(&sm.v_full[slot], slot_parity, &sm.abort_flag, wait_limit)) { ok = false; break; }
     const uint32_t v_lo = kv_lo + slot * (kTileBytes >> 4);
     const uint32_t acc_first = (dsc & kTileFirst) ? 0u : 1u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag)) { ok = false; break; }
-      TRACE(g, 3 + h);
+      if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag, wait_limit)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < kHalf / 16; ++ks) {
@@ -559,37 +592,53 @@ __device__ void mma_pv_role(Shared& sm, const Params& p, unsigned char* sKV, uin
     if (!ok) break;
     if (leader) {
       mma_commit(&sm.v_empty[slot]);
-      mma_commit(&sm.pv_done[b]);
+      // (test hook: a withheld completion signal makes the bounded waits on it run out)
+      if ((int)g != p.withhold_tile) mma_commit(&sm.pv_done[b]);
     }
-    TRACE(g, 5);
     ++g;
     if (++slot == kVStages) { slot = 0; slot_parity ^= 1; }
   }
   if (!ok && leader) flag_abort(sm, p, 301);
+  __syncwarp();
+  if (sm.abort_flag) drain_mmas(sm, &sm.mma_drain[1], leader, wait_limit);
 }
 
 // ------------------------------------------------------------------------------------------------
 // softmax + correction + epilogue: two warpgroups of 128 threads; thread = query row, warpgroup h
-// owns key columns [64h, 64h+64) of every tile.
-__device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, int warp_in_group, int lane) {
+// owns key columns [kHalf h, kHalf (h+1)) of every tile.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t* r) {   // N columns, N a multiple of 32
+#pragma unroll
+  for (int c = 0; c < N; c += 32) tmem_ld_32x32b_x32(taddr + c, *reinterpret_cast<uint32_t(*)[32]>(r + c));
+}
+
+template <class C>
+__device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int h, int warp_in_group, int lane) {
+  constexpr int kD = C::kD, kBlk = C::kBlk, kHalf = C::kHalf;
+  constexpr int kOutCh = kD / 2;                             // output channels written by one warpgroup
   const unsigned full = 0xffffffffu;
+  const long long wait_limit = p.wait_limit;
   const uint32_t lane_base = tmem + ((uint32_t)(warp_in_group * 32) << 16);
   const uint32_t t_o = lane_base + kTmemO + h * kD;          // this group's accumulator
   const uint32_t t_o_other = lane_base + kTmemO + (1 - h) * kD;
   const int row = warp_in_group * 32 + lane;
   const float sl2 = p.scale * 1.4426950408889634f;
   uint32_t g = 0, n_merge = 0;
+  uint32_t n_item = 0, g_item0 = 0;        // item trace only
   float m_used = -INFINITY, l = 0.f;
-  Cursor cur;
+  Cursor<C> cur;
   PROF_DECL
   auto release = [&](uint32_t r) {
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.rec_empty[r]);
   };
+  // A wait that gives up must give up for the whole warp: the loop holds warp-synchronising
+  // operations (TMEM loads and stores, votes), so the lanes leave together or not at all.
+#define SWAIT(bar, parity, slot) __all_sync(full, WAIT(bar, parity, slot))
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, PROF_ACC(0), release);                    // prof 0: no record yet
+    const uint32_t dsc = next_desc(sm, cur, wait_limit, PROF_ACC(0), release);        // prof 0: no record yet
+    if (__any_sync(full, dsc == kDescAbort)) { flag_abort(sm, p, 400); break; }
     if (dsc == kDescStop) break;
-    if (dsc == kDescAbort) { flag_abort(sm, p, 400); break; }
     const bool first = (dsc & kTileFirst) != 0;
 
     if (!(dsc & kTileEnd)) {
@@ -598,17 +647,14 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       const bool approx = (dsc & kTileApprox) != 0;
       const int cols_valid = approx ? kBlk : min(kBlk, p.N - (int)(dsc >> 5));
       const bool general = approx || cols_valid < kBlk;
-      if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
+      if (!SWAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }  // prof 1: S not ready
       tc_fence_after();
-      if (row == 0) TRACE(g, 6 + 3 * h);
-      WTRACE(0);
-      // ---- this group's half row of S (64 fp32) into registers with one wait
+      if (first && warp_in_group == 0 && lane == 0) { ITRACE(n_item, h ? 11 : 5); g_item0 = g; }
+      // ---- this group's half row of S (kHalf fp32) into registers with one wait
       uint32_t sr[kHalf];
       PROF_T0
-      tmem_ld_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
-      tmem_ld_32x32b_x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+      tmem_ld_cols<kHalf>(t_s, sr);
       tmem_ld_wait();
-      WTRACE(1);
       PROF_ADD(7)                                                                      // prof 7: loading S
       if (general) {
         // bring the rare tiles (approximate chunk, ragged last block) to the common form
@@ -631,13 +677,14 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       }
       float mx;
       {
+        constexpr int kQ = kHalf / 4;
         float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < kQ; ++c) {
           m0 = fmaxf(m0, __uint_as_float(sr[c]));
-          m1 = fmaxf(m1, __uint_as_float(sr[16 + c]));
-          m2 = fmaxf(m2, __uint_as_float(sr[32 + c]));
-          m3 = fmaxf(m3, __uint_as_float(sr[48 + c]));
+          m1 = fmaxf(m1, __uint_as_float(sr[kQ + c]));
+          m2 = fmaxf(m2, __uint_as_float(sr[2 * kQ + c]));
+          m3 = fmaxf(m3, __uint_as_float(sr[3 * kQ + c]));
         }
         mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * sl2;       // -inf when the whole half is masked
       }
@@ -650,10 +697,10 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         const float f = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
         PROF_COUNT(4);                                                                  // prof 4: number of rescales
         // P V of the previous tile must have landed in O_h
-        if (!WAIT(&sm.pv_done[b ^ 1], ((g - 1) >> 1) & 1, 2)) { flag_abort(sm, p, 402); break; }
+        if (!SWAIT(&sm.pv_done[b ^ 1], ((g - 1) >> 1) & 1, 2)) { flag_abort(sm, p, 402); break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < kD / 32; ++c) {
           uint32_t o[32];
           tmem_ld_32x32b_x32(t_o + c * 32, o);
           tmem_ld_wait();
@@ -664,7 +711,6 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
         l *= f;
         m_used = m_new;
       }
-      WTRACE(2);
       // ---- P = exp2(sl2 * S - m) (scaling and row sum as packed fp32 pairs); P (bf16) back to
       //      TMEM over the start of the half
       {
@@ -688,19 +734,14 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
           const float2 t = __fadd2_rn(s_a, s_b);
           l += t.x + t.y;
         }
-        tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+        if constexpr (kHalf == 64) tmem_st_32x32b_x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+        else tmem_st_32x32b_x16(t_s, *reinterpret_cast<uint32_t(*)[16]>(&sr[0]));
       }
       PROF_ADD(8)                                                                      // prof 8: load + arithmetic
-      if (row == 0) TRACE(g, 7 + 3 * h);
-      WTRACE(3);
       tmem_st_wait();
-      WTRACE(4);
       tc_fence_before();
       __syncwarp();                                  // one arrival per warp: 4 instead of 128 on the barrier
       if (lane == 0) mbar_arrive(&sm.p_full[h][b]);
-      if (row == 0) TRACE(g, 8 + 3 * h);
-      if (lane == 0) TRACE(g, 16 + 4 * h + warp_in_group);
-      WTRACE(5);
       PROF_ADD(9)                                                                      // prof 9: whole tile
 #ifdef SOL_PROFILE
       if (approx) { prof.v[10] += clock64() - prof_t0; ++prof.v[0]; }                  // prof 10 / 0: approximate tiles: cycles / count
@@ -714,27 +755,33 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
     const int q_row = cur.rec->q_row;
     const int q_rows = min(kBlk, p.N - q_row);
     __nv_bfloat16* orow = p.out + (size_t)cur.rec->b * (size_t)p.st.batch + (size_t)cur.rec->h * (size_t)p.st.head +
-                          (size_t)(q_row + row) * (size_t)p.st.row + h * kHalf;
+                          (size_t)(q_row + row) * (size_t)p.st.row + h * kOutCh;
     PROF_T0
+    if (warp_in_group == 0 && lane == 0) {
+      ITRACE(n_item, h ? 12 : 6);
+      if (h == 0) ITRACE_VAL(n_item, 10, (long long)(g - g_item0));
+    }
     if (!(dsc & kTileEmptyItem)) {
       // the last P V of the item (one commit covers both halves)
-      if (!WAIT(&sm.pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, 3)) { flag_abort(sm, p, 403); break; }   // prof 3
+      if (!SWAIT(&sm.pv_done[(g - 1) & 1], ((g - 1) >> 1) & 1, 3)) { flag_abort(sm, p, 403); break; }   // prof 3
       tc_fence_after();
+      if (h == 0 && warp_in_group == 0 && lane == 0) ITRACE(n_item, 7);
       sm.ml[h][row] = make_float2(m_used, l);
       mbar_arrive(&sm.x_full);
-      if (!WAIT(&sm.x_full, n_merge & 1, 6)) { flag_abort(sm, p, 404); break; }       // prof 6: other group not done
+      if (!SWAIT(&sm.x_full, n_merge & 1, 6)) { flag_abort(sm, p, 404); break; }      // prof 6: other group not done
+      if (warp_in_group == 0 && lane == 0) ITRACE(n_item, h ? 13 : 8);
       const float2 other = sm.ml[1 - h][row];
       const float m = fmaxf(m_used, other.x);
       const float w_own = (m_used == -INFINITY) ? 0.f : ex2(m_used - m);
       const float w_other = (other.x == -INFINITY) ? 0.f : ex2(other.x - m);
       const float inv = 1.f / (l * w_own + other.y * w_other);
       const float c_own = w_own * inv, c_other = w_other * inv;
-      // this thread writes channels [64h, 64h+64) of its row
+      // this thread writes channels [kOutCh h, kOutCh (h+1)) of its row
 #pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < kOutCh / 32; ++c) {
         uint32_t a[32], bb[32];
-        tmem_ld_32x32b_x32(t_o + h * kHalf + c * 32, a);
-        tmem_ld_32x32b_x32(t_o_other + h * kHalf + c * 32, bb);
+        tmem_ld_32x32b_x32(t_o + h * kOutCh + c * 32, a);
+        tmem_ld_32x32b_x32(t_o_other + h * kOutCh + c * 32, bb);
         tmem_ld_wait();
         if (row < q_rows) {
 #pragma unroll
@@ -760,19 +807,23 @@ __device__ void softmax_role(Shared& sm, const Params& p, uint32_t tmem, int h, 
       // neither group may start the next item (whose first P V overwrites O0 / O1) before both
       // have finished reading
       mbar_arrive(&sm.x_done);
-      if (!WAIT(&sm.x_done, n_merge & 1, 6)) { flag_abort(sm, p, 405); break; }
+      if (!SWAIT(&sm.x_done, n_merge & 1, 6)) { flag_abort(sm, p, 405); break; }
+      if (warp_in_group == 0 && lane == 0) ITRACE(n_item, h ? 14 : 9);
       ++n_merge;
     } else if (row < q_rows) {
       // a query block that routed nothing in keep-or-drop mode has no attention mass at all
-      for (int c = 0; c < kHalf; c += 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
+      for (int c = 0; c < kOutCh; c += 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
     }
     m_used = -INFINITY;
     l = 0.f;
+    ++n_item;
     PROF_ADD(2)                                                                        // prof 2: whole epilogue
   }
-  if (lane == 0 && warp_in_group == 0 && h == 0) PROF_FLUSH(3);
+#undef SWAIT
+  if (lane == 0 && warp_in_group == 0 && h == 0) { PROF_FLUSH(3); CTATRACE(3, prof::gtimer()); }
 }
 
+template <class C>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kc,
@@ -780,8 +831,8 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char* sQ = base;
-  unsigned char* sKV = base + kTileBytes;
-  Shared& sm = *reinterpret_cast<Shared*>(base + kTileBytes + kStages * kTileBytes);
+  unsigned char* sKV = base + C::kQBytes;
+  Shared<C>& sm = *reinterpret_cast<Shared<C>*>(base + C::kQBytes + (kKStages + kVStages) * C::kTileBytes);
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
@@ -799,6 +850,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     mbar_init(&sm.x_full, 256); mbar_init(&sm.x_done, 256);
     mbar_init(&sm.kc_full[0], 1); mbar_init(&sm.kc_full[1], 1);
+    mbar_init(&sm.mma_drain[0], 1); mbar_init(&sm.mma_drain[1], 1);
     fence_mbar_init();
   }
   if (warp == kWarpProducer && lane == 0) {
@@ -812,73 +864,85 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem = sm.tmem_base;
 
   if (warp < 8) {
-    softmax_role(sm, p, tmem, warp / 4, warp % 4, lane);
+    softmax_role<C>(sm, p, tmem, warp / 4, warp % 4, lane);
   } else if (warp == kWarpRouter) {
-    router_role(sm, p, lane);
+    router_role<C>(sm, p, lane);
   } else if (warp == kWarpProducer) {
-    if (lane == 0) producer_role(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
+    if (lane == 0) producer_role<C>(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
   } else if (warp == kWarpQK) {
-    mma_qk_role(sm, p, sQ, sKV, tmem);
+    mma_qk_role<C>(sm, p, sQ, sKV, tmem);
   } else {
-    mma_pv_role(sm, p, sKV, tmem);
+    mma_pv_role<C>(sm, p, sKV, tmem);
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-}  // namespace
+// Test hook (sol_attn_debug_set_wait): the wait limit and the withheld tile of the following launches.
+long long g_wait_limit = kWaitCycles;
+int g_withhold_tile = -1;
 
-#ifdef SOL_PROFILE
-}  // namespace sol
-// Debug builds only: copies the per-CTA, per-role wait-cycle counters of the last launch to the host.
-extern "C" int sol_attn_debug_profile(long long* host_out, int n_values) {
-  const size_t total = sizeof(long long) * sol::kProfCtas * sol::kProfRoles * sol::kProfSlots;
-  const size_t want = sizeof(long long) * (size_t)n_values;
-  return (int)cudaMemcpyFromSymbol(host_out, sol::g_prof, want < total ? want : total);
-}
-extern "C" int sol_attn_debug_trace(long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, sol::g_trace, sizeof(long long) * sol::kTraceTiles * sol::kTraceEvents);
-}
-namespace sol {
-#endif
-
-bool fwd_sm100_supports(const Problem& p) { return p.d == kD && p.block_q == kBlk && p.block_k == kBlk; }
-
-cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k,
-                             const __nv_bfloat16* v, __nv_bfloat16* out, const WsPtrs& ws, const float* tau,
-                             int32_t* counts, uint32_t* mask_out, cudaStream_t stream,
-                             int* n_launches) {
+template <class C>
+cudaError_t launch_instance(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                            __nv_bfloat16* out, const WsPtrs& ws, const float* tau, int32_t* counts, uint32_t* mask_out,
+                            cudaStream_t stream, int* n_launches) {
   CUtensorMap tq, tk, tv, tkc, tvm;
   bool rows_inner = true, pooled_inner = true;
-  auto user_map = [&](CUtensorMap* m, const void* base) {
-    return make_tmap_bf16_4d(m, base, p.B, p.H, p.N, kD, kBlk, p.st.row, p.st.head, p.st.batch, &rows_inner);
+  auto user_map = [&](CUtensorMap* m, const void* base, int box_rows) {
+    return make_tmap_bf16_4d(m, base, p.B, p.H, p.N, C::kD, box_rows, p.st.row, p.st.head, p.st.batch, &rows_inner);
   };
   auto pooled_map = [&](CUtensorMap* m, const void* base) {      // dense [B][H][Nk][d]
-    return make_tmap_bf16_4d(m, base, p.B, p.H, p.Nk, kD, kBlk, kD, (long long)p.Nk * kD, (long long)p.H * p.Nk * kD,
-                             &pooled_inner);
+    return make_tmap_bf16_4d(m, base, p.B, p.H, p.Nk, C::kD, C::kBlk, C::kD, (long long)p.Nk * C::kD,
+                             (long long)p.H * p.Nk * C::kD, &pooled_inner);
   };
-  if (!user_map(&tq, q) || !user_map(&tk, k) || !user_map(&tv, v) || !pooled_map(&tkc, ws.kcb) ||
-      !pooled_map(&tvm, ws.vmb) || !pooled_inner)
+  if (!user_map(&tq, q, kRowsQ) || !user_map(&tk, k, C::kBlk) || !user_map(&tv, v, C::kBlk) ||
+      !pooled_map(&tkc, ws.kcb) || !pooled_map(&tvm, ws.vmb) || !pooled_inner)
     return cudaErrorInvalidValue;
   Params prm{};
   prm.qbar = ws.qbar; prm.kc = ws.kc; prm.tau = tau; prm.out = out; prm.counts = counts; prm.mask_out = mask_out;
   prm.status = ws.status; prm.N = p.N; prm.Nq = p.Nq; prm.Nk = p.Nk; prm.total_work = p.BH * p.Nq;
   prm.mode = p.mode; prm.scale = p.scale; prm.forced = p.forced;
   prm.st = p.st; prm.rows_inner = rows_inner ? 1 : 0;
+  prm.wait_limit = g_wait_limit; prm.withhold_tile = g_withhold_tile;
 
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const size_t smem = 1024 + kTileBytes + kStages * kTileBytes + sizeof(Shared);
-  e = cudaFuncSetAttribute(fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = 1024 + C::kQBytes + (kKStages + kVStages) * C::kTileBytes + sizeof(Shared<C>);
+  e = cudaFuncSetAttribute(fwd_sm100_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int grid = prm.total_work < sms ? prm.total_work : sms;
-  fwd_sm100_kernel<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
+  fwd_sm100_kernel<C><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
   if (n_launches) *n_launches += 1;
   return cudaGetLastError();
+}
+
+}  // namespace
+
+bool fwd_sm100_supports(const Problem& p) {
+  return (p.d == 64 || p.d == 128) && p.block_q == p.block_k && (p.block_k == 64 || p.block_k == 128);
+}
+
+void fwd_sm100_set_wait(long long wait_cycles, int withhold_tile) {
+  g_wait_limit = wait_cycles > 0 ? wait_cycles : kWaitCycles;
+  g_withhold_tile = withhold_tile;
+}
+
+cudaError_t launch_fwd_sm100(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                             const __nv_bfloat16* v, __nv_bfloat16* out, const WsPtrs& ws, const float* tau,
+                             int32_t* counts, uint32_t* mask_out, cudaStream_t stream,
+                             int* n_launches) {
+  if (!fwd_sm100_supports(p)) return cudaErrorInvalidValue;
+  if (p.d == 128 && p.block_k == 128)
+    return launch_instance<Cfg<128, 128>>(p, q, k, v, out, ws, tau, counts, mask_out, stream, n_launches);
+  if (p.d == 64 && p.block_k == 64)
+    return launch_instance<Cfg<64, 64>>(p, q, k, v, out, ws, tau, counts, mask_out, stream, n_launches);
+  if (p.d == 128)
+    return launch_instance<Cfg<128, 64>>(p, q, k, v, out, ws, tau, counts, mask_out, stream, n_launches);
+  return launch_instance<Cfg<64, 128>>(p, q, k, v, out, ws, tau, counts, mask_out, stream, n_launches);
 }
 
 }  // namespace sol

@@ -44,17 +44,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait on an mbarrier phase.  Gives up after ~kWaitCycles SM clocks or as soon as
-// another thread of the CTA has flagged an abort; returns false in that case.
+// Bounded wait on an mbarrier phase.  Gives up after ~`limit` SM clocks (kWaitCycles unless the
+// caller says otherwise) or as soon as another thread of the CTA has flagged an abort; returns
+// false in that case.
 constexpr long long kWaitCycles = 4000000000LL;   // about 2-3 s of SM clocks
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0x3ffu) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
   return true;

@@ -437,3 +437,33 @@ def test_cuda_graph_capture_and_replay(impl):
     eager2, counts2, _, _ = hp.run_gpu(q, k, v, 128, 0.6, impl=_impl(impl), want_mask=False)
     assert torch.equal(out.view(torch.int16), eager2.view(torch.int16))
     assert torch.equal(ws.counts, counts2)
+
+
+# ----------------------------------------------------------------------------- device-side failure path
+def test_bounded_wait_runs_out_and_the_next_call_is_clean():
+    """Every wait inside the tcgen05 kernel has a limit.  With the limit shortened to about a millisecond
+    and one "value GEMM finished" signal per CTA withheld (a testing hook of the library: nothing faults,
+    traps or spins unbounded), the waits on that signal run out, the CTA drains its copies and MMAs,
+    releases TMEM and returns; the host reads SOL_ERR_DEVICE_TIMEOUT from the status word.  The same
+    workspace then serves a normal call whose result matches the oracle."""
+    bits = _small_problem(71, 1, 2, 1536, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    ws = sb.make_workspace(1, 2, 1536, 128, 128, 128)
+    out = torch.empty_like(q)
+    sb.sol_attn_debug_set_wait(2_000_000, 1)
+    try:
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.2, impl=sb.SOL_IMPL_TCGEN05)
+        torch.cuda.synchronize()
+        detail = int(ws.buf[:8].view(torch.int32)[1].item())
+        sb.sol_attn_bind_workspace(ws)
+        st = sb.sol_attn_read_device_status()
+    finally:
+        sb.sol_attn_debug_set_wait(0, -1)
+    assert st == sb.SOL_ERR_DEVICE_TIMEOUT, sb.status_string(st)
+    assert detail != 0                                       # where the first wait gave up
+    assert sb.sol_attn_read_device_status() == sb.SOL_OK      # reading the status clears it
+    out2, counts, mask, _ = hp.run_gpu(q, k, v, 128, 0.2, impl=sb.SOL_IMPL_TCGEN05, ws=ws)
+    o = hp.dev_to_f64(out2)
+    for h in range(2):
+        hp.check_head(synth.widen(bits[0][0, h], np.float64), synth.widen(bits[1][0, h], np.float64),
+                      synth.widen(bits[2][0, h], np.float64), o[0, h], mask[0, h], counts[0, h].cpu().numpy(), 128, 0.2)
