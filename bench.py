@@ -17,8 +17,10 @@ one batch (B=1, H=40, N=75600, d=128, block 128 for the default workload).  Prin
 * cpu_baseline: the CPU oracle timed on a bounded sample of the same workload.
 * sweep: every density of the workload's threshold sweep plus the dense-mode run.
 
-Under torchrun every rank runs the same workload on its own GPU (heads are independent; there
-is no collective in the operator), timing is max over ranks and ``value`` is the aggregate.
+Under torchrun ONE call is sharded by heads: rank r generates and processes only its own contiguous
+range of the workload's heads (heads are independent; there is no collective on the data path), timing
+is max over ranks and ``value`` is the whole job's dense-equivalent throughput (``scaling``: strong).
+``--replicas`` makes every rank run the whole workload instead (weak scaling).
 ``--impl reference`` times the CPU oracle (rank 0 only).
 """
 from __future__ import annotations
@@ -38,6 +40,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2607_24027_b200 import synth  # noqa: E402
 from paper_2607_24027_b200.configs import DENSITY_SWEEP, WORKLOADS, load_betas  # noqa: E402
+from paper_2607_24027_b200.shard import head_partition  # noqa: E402
 
 METRIC = "dense-equivalent attention throughput at 720p (ms/call in ms_per_step)"
 UNIT = "TFLOP/s (dense-equivalent)"
@@ -52,18 +55,32 @@ def load_peaks():
     return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
+def measured_traffic(kernel, wl, n_heads):
+    """DRAM bytes of one launch of `kernel`, from the ncu summary committed under profiles/ (written by
+    ``python -m paper_2607_24027_b200.ncu_summary``): a small-case capture scaled by the head count
+    (every tensor crosses HBM once per launch, so traffic grows with the heads).  None when no summary
+    covers this workload."""
+    path = os.path.join(ROOT, "profiles", f"{kernel}_{wl.name}.json")
+    if not os.path.exists(path):
+        return None, None
+    rec = json.load(open(path))
+    per_head = (rec["dram_bytes_read"] + rec["dram_bytes_write"]) / float(rec["heads"])
+    return per_head * n_heads, {"file": os.path.relpath(path, ROOT), "captured_heads": rec["heads"],
+                                "kernel_git_hash": rec.get("kernel_git_hash")}
+
+
 def dense_flops(wl):
     return 4.0 * wl.batch * wl.heads * float(wl.seq_len) ** 2 * wl.d
 
 
-def computed_flops(wl, counts_sum, mode_dense=False):
+def computed_flops(wl, counts_sum, mode_dense=False, n_bh=None):
     """Algorithmic FLOPs of one fused-kernel launch: routed (query block, key block) pairs are
     4*b*b*d each; the approximate outer loop is a b x Nk x d pair of GEMMs per query block."""
     b, d, nk = wl.block, wl.d, wl.n_blocks
     exact = float(counts_sum) * 4.0 * b * b * d
     if mode_dense:
         return exact
-    approx = wl.batch * wl.heads * float(nk) * 4.0 * b * nk * d
+    approx = (wl.batch * wl.heads if n_bh is None else n_bh) * float(nk) * 4.0 * b * nk * d
     return exact + approx
 
 
@@ -124,26 +141,31 @@ class ClockSampler:
 _HEAD0 = {}
 
 
-def oracle_sample(wl, beta, n_tiles=6, seed=0):
-    """Time the oracle on a bounded sample: routing of head 0 plus `n_tiles` query blocks of it
-    (Algorithm 1).  Returns (seconds per query block incl. its share of routing, description)."""
-    from oracle import sol_attn_oracle as orc
+def _head0(wl):
     if wl.name not in _HEAD0:                 # input generation is not part of the timed work
         qb, kb, vb = synth.generate(wl, heads=slice(0, 1))
         _HEAD0[wl.name] = tuple(synth.widen(x[0], np.float64) for x in (qb, kb, vb))
-    q, k, v = _HEAD0[wl.name]
+    return _HEAD0[wl.name]
+
+
+def oracle_head_slice(wl, beta, step, n_steps):
+    """Time the oracle on the pre-attention step of head 0 plus the query blocks i = step (mod n_steps)
+    of that head (Algorithm 1); n_steps = 1 is the whole head.  Returns (seconds extrapolated to the
+    whole head, description, achieved density)."""
+    from oracle import sol_attn_oracle as orc
+    q, k, v = _head0(wl)
     t0 = time.perf_counter()
     r = orc.routing(q, k, v, wl.block, wl.block, beta)
     t_route = time.perf_counter() - t0
     nq = r.mask.shape[0]
-    rng = np.random.default_rng(seed)
-    tiles = sorted(rng.choice(nq, size=min(n_tiles, nq), replace=False).tolist())
+    tiles = list(range(step % n_steps, nq, n_steps))
     t0 = time.perf_counter()
     orc.sol_attn_streaming(q, k, v, r.kc, r.vc, r.tau, wl.block, wl.block, chunk=16, q_tiles=tiles)
     t_tiles = time.perf_counter() - t0
-    per_tile = t_tiles / len(tiles) + t_route / nq
-    return per_tile, f"head 0: routing of all {nq} query blocks + Algorithm 1 on query blocks {tiles}", \
-        float(r.mask.mean())
+    t_head = t_route + t_tiles * nq / len(tiles)
+    what = (f"head 0 of {wl.batch * wl.heads}: pooling + thresholds of all {nq} query blocks, Algorithm 1 on "
+            f"{len(tiles)} of them" + ("" if n_steps == 1 else f" (every {n_steps}th, offset by the step)"))
+    return t_head, what, float(r.mask.mean())
 
 
 def cpu_threads():
@@ -156,25 +178,31 @@ def cpu_threads():
 
 
 def run_reference(args, wl, beta):
+    """The reference arm of this build is the CPU oracle, as it stands, on the host cores.  A whole 720p
+    call is hours of float64 numpy, so each step times a bounded sample -- the pre-attention step of head 0
+    and every K-th query block of it, K = the number of steps, so that the timed steps together cover the
+    head once -- and extrapolates: x (blocks / sampled blocks) to the head, x heads to the call."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    total_tiles = wl.batch * wl.heads * wl.n_blocks
+    n_bh = wl.batch * wl.heads
     times = []
     sample = ""
+    n_slices = max(1, args.steps)
     for step in range(args.warmup + args.steps):
-        per_tile, sample, _ = oracle_sample(wl, beta, n_tiles=4, seed=step)
+        t_head, sample, _ = oracle_head_slice(wl, beta, step, n_slices)
         if step >= args.warmup:
-            times.append(per_tile * total_tiles)
+            times.append(t_head * n_bh)
     t = float(np.mean(times))
     val = dense_flops(wl) / t / 1e12
+    note = f"{sample}; 1 head x {n_bh}, extrapolated"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "scaling": "strong", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": f"{wl.name} density {args.density}", "B": wl.batch, "H": wl.heads,
                        "N": wl.seq_len, "d": wl.d, "block": wl.block, "beta": beta,
-                       "note": "each step times a bounded sample and extrapolates by query-block count"},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+                       "extrapolated": note},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": note},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -222,6 +250,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--heads", type=int, default=0, help="override the head count (profiling small cases)")
+    ap.add_argument("--replicas", action="store_true",
+                    help="multi-GPU: every rank runs the whole workload (weak scaling) instead of a head shard")
     args = ap.parse_args()
 
     wl = WORKLOADS[args.workload]
@@ -253,8 +283,17 @@ def main():
 
     # inputs: generated on the host by the seeded generator, then kept resident in HBM
     import dataclasses
-    wl_rank = dataclasses.replace(wl, seed=wl.seed + 1000 * rank) if rank else wl
-    qb, kb, vb = synth.generate(wl_rank)
+    if world > 1 and not args.replicas:
+        # one call sharded by heads: this rank's contiguous range of (batch, head) pairs, nothing else
+        mine = head_partition(wl.batch * wl.heads, world, rank)
+        qb, kb, vb = (x[None] for x in synth.generate(wl, heads=mine))       # [1, n_local, N, d]
+        if qb.shape[1] == 0:
+            raise SystemExit(f"rank {rank} of {world} owns no head of {wl.batch * wl.heads}")
+        job_flops = dense_flops(wl)                                           # the whole job, whatever N
+    else:
+        wl_rank = dataclasses.replace(wl, seed=wl.seed + 1000 * rank) if rank else wl
+        qb, kb, vb = synth.generate(wl_rank)
+        job_flops = world * dense_flops(wl)
     to_dev = lambda x: torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16)
     q, k, v = to_dev(qb), to_dev(kb), to_dev(vb)
     out = torch.empty_like(q)
@@ -307,7 +346,7 @@ def main():
     def pool_kv_only():                      # the pooling kernel alone (no thresholds): K and V
         sb.sol_attn_pool(None, k, v, wl.block, wl.block, beta)
 
-    dflops = dense_flops(wl)
+    dflops = 4.0 * B * H * float(N) ** 2 * d          # dense-equivalent work of THIS rank's heads
     peaks = load_peaks()
 
     # ---- headline: whole path, inputs resident
@@ -321,7 +360,7 @@ def main():
 
     # ---- fused kernel alone (workspace already holds the pre-attention results)
     ms_kernel = timed(kernel_only, args.steps, 1)
-    cflops = computed_flops(wl, counts_sum)
+    cflops = computed_flops(wl, counts_sum, n_bh=B * H)
     achieved = cflops / (ms_kernel * 1e-3) / 1e12
     ms_pool = timed(pool_only, args.steps, 1)
     ms_pool_kv = timed(pool_kv_only, args.steps, 1)
@@ -356,7 +395,7 @@ def main():
             cs = int(ws.counts.sum().item())
             ms_k = timed(lambda: kernel_only(b), max(3, args.steps // 2), 1)
             dens = cs / float(B * H * wl.n_blocks * wl.n_blocks)
-            cf = computed_flops(wl, cs)
+            cf = computed_flops(wl, cs, n_bh=B * H)
             sweep.append({"mode": "sol", "target_density": rho, "beta": b, "density": dens,
                           "ms_per_call": ms_f, "kernel_ms": ms_k, "dense_equiv_tflops": dflops / ms_f / 1e9,
                           "computed_tflops": cf / ms_k / 1e9,
@@ -380,7 +419,14 @@ def main():
                                                                tau_b, order=order, counts=cnt_b), args.steps, 1)
         ms_topp = timed(lambda: sb.sol_attn_route_materialized(ws.qbar, ws.kc, sb.SOL_ROUTE_TOPP, 0.9, pmap,
                                                                tau_b, order=order, counts=cnt_b), args.steps, 1)
-        routing = {"thresholds_ms": ms_thr, "topk_ms": ms_topk, "topp_ms": ms_topp,
+        mu_s, sg_s, tau_s = (torch.empty(B, H, nb, device="cuda") for _ in range(3))
+        ms_thr_static = None
+        if B * H * d * (d + 1) <= sb.sol_attn_thresholds_static_max_floats():
+            qbar_c, kc_c = ws.qbar.contiguous(), ws.kc.contiguous()
+            ms_thr_static = timed(lambda: sb.sol_attn_thresholds_static(qbar_c, kc_c, beta, mu_s, sg_s, tau_s),
+                                  args.steps, 1)
+        routing = {"thresholds_ms": ms_thr, "thresholds_static_ms": ms_thr_static,
+                   "topk_ms": ms_topk, "topp_ms": ms_topp,
                    "topk_over_thresholds": ms_topk / ms_thr, "topp_over_thresholds": ms_topp / ms_thr,
                    "materialised_bytes": int(pmap.numel() * 4 + order.numel() * 4),
                    "note": "thresholds: mean, covariance and tau kernels on pooled data (nothing of size Nq x Nk "
@@ -404,37 +450,48 @@ def main():
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only)
     cpu = None
     if world == 1 and not args.no_cpu:
-        per_tile, sample, _ = oracle_sample(wl, beta, n_tiles=6)
-        t_cpu = per_tile * B * H * wl.n_blocks
+        t_head, sample, _ = oracle_head_slice(wl, beta, 0, 1)          # one whole head, timed once
+        t_cpu = t_head * B * H
         cpu = {"value": dflops / t_cpu / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-               "sample": sample + f"; {per_tile:.3f} s per query block, extrapolated x{B * H * wl.n_blocks}"}
+               "sample": sample + f"; {t_head:.1f} s for the head; 1 head x {B * H}, extrapolated"}
 
+    traffic, traffic_src = measured_traffic("fwd_sm100_kernel" if args.kernel != "mma_sync" else "fwd_mma_sync_kernel",
+                                            wl, B * H)
     line = {
-        "metric": METRIC, "value": world * dflops / (ms_step * 1e-3) / 1e12, "unit": UNIT,
+        "metric": METRIC, "value": job_flops / (ms_step * 1e-3) / 1e12, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "higher_is_better": True, "scaling": "weak" if (args.replicas or world == 1) else "strong",
+        "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"{wl.name} density {args.density}", "B": B, "H": H, "N": N, "d": d,
                    "block": wl.block, "beta": beta, "achieved_density": density, "kernel": args.kernel,
                    "l2": "inputs (3 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
-                   "parallelism": "replicas (no collective)" if world > 1 else "single GPU"},
+                   "parallelism": ("single GPU" if world == 1 else "replicas (no collective)" if args.replicas else
+                                   f"one call sharded by heads: {H} of {wl.batch * wl.heads} heads on this rank, "
+                                   "no collective on the data path")},
         "clocks": clk.summary(),
-        "e2e": {"value": world * dflops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
-                "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": q.numel() * 2},
+        "e2e": {"value": job_flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+                # all ranks together: every rank copies its own q, k, v in and its own output back
+                "h2d_bytes_per_step": 3 * q.numel() * 2 * (world if args.replicas else 1) if world == 1 or args.replicas
+                else 3 * wl.batch * wl.heads * N * d * 2,
+                "d2h_bytes_per_step": q.numel() * 2 * (world if args.replicas else 1) if world == 1 or args.replicas
+                else wl.batch * wl.heads * N * d * 2},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "fwd_sm100_kernel" if args.kernel != "mma_sync" else "fwd_mma_sync_kernel",
                      "achieved": achieved, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_burst"], "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": (achieved / peaks["bf16_sustained"]) if peaks["bf16_sustained"] else None,
                      "kernel_ms": ms_kernel, "computed_flops": cflops,
-                     # dram__bytes_read + dram__bytes_write of one launch, from the 4-head ncu capture
-                     # (298 MB) scaled by the head count: every tensor crosses HBM once per launch
-                     "traffic": 298.4e6 / 4.0 * H * B if wl.name == "video720" else None},
-        "pool": {"bound": "hbm", "kernel": "pool_kernel", "ms": ms_pool_kv,
-                 "achieved": pool_bytes / (ms_pool_kv * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                 "frac": pool_bytes / (ms_pool_kv * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                 "note": "pooling kernel alone on K and V (2 of the 3 tensors; q is pooled by the same kernel)",
-                 "pre_attention_ms": ms_pool},
+                     # dram__bytes_read + dram__bytes_write of one launch, read from the ncu summary under
+                     # profiles/ (a small-case capture scaled by the head count)
+                     "traffic": traffic, "traffic_source": traffic_src,
+                     # the HBM-bound pre-pass: the pooling kernel alone on K and V (2 of the 3 tensors; q is
+                     # pooled by the same kernel), bytes = K + V read once + their pooled copies written
+                     "pool": {"bound": "hbm", "kernel": "pool_kernel", "ms": ms_pool_kv, "bytes": pool_bytes,
+                              "achieved": pool_bytes / (ms_pool_kv * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                              "unit": "GB/s", "frac": pool_bytes / (ms_pool_kv * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                              "pre_attention_ms": ms_pool},
+                     "pool_frac": pool_bytes / (ms_pool_kv * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "cpu_baseline": cpu,
         "sweep": sweep,
         "ablation": ablation,

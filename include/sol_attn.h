@@ -25,7 +25,7 @@
  *     overwritten by every call.  Calls that share a workspace and overlap on the GPU race.
  *   - Supported shapes: d in {64, 128}; block_q == block_k in {64, 128} for the fused
  *     kernels (the pooling pre-pass accepts any block size in [1, 1024]); B, H, N >= 1;
- *     ceil(N / block_k) <= 65535.  Anything else returns SOL_ERR_UNSUPPORTED_SHAPE.
+ *     ceil(N / block_k) <= 65535; B * H <= 65535.  Anything else returns SOL_ERR_UNSUPPORTED_SHAPE.
  */
 #ifndef SOL_ATTN_H_
 #define SOL_ATTN_H_
@@ -48,7 +48,8 @@ enum {
   SOL_ERR_WORKSPACE         = -4,  /* no workspace bound / workspace too small or misaligned   */
   SOL_ERR_CUDA              = -5,  /* a CUDA runtime or driver call failed (launch, tensor map)*/
   SOL_ERR_DEVICE_TIMEOUT    = -6,  /* a bounded device-side wait expired; output is invalid    */
-  SOL_ERR_SCRATCH_LIMIT     = -7   /* problem larger than the library's built-in scratch array */
+  SOL_ERR_SCRATCH_LIMIT     = -7,  /* problem larger than the library's built-in scratch array */
+  SOL_ERR_STATIC_SCRATCH    = -8   /* the built-in scratch array could not be set up on this device */
 };
 
 /* what the fused kernel computes */
@@ -194,8 +195,8 @@ sol_status_t sol_attn_read_device_status(sol_stream_t stream);
  * another framework's memory pool, a process whose device memory was reserved up front, a
  * serving loop in which an allocation would synchronise the device.  Such callers cannot provide
  * the workspace the other entry points keep the pooled-key moments in, so here the moments live
- * in a fixed array inside the library image: 4 MiB of device memory on every GPU that loads the
- * library, from load until exit.
+ * in a fixed array inside the library image: 4 MiB of device memory on every GPU that has made its
+ * first call (see below), held until the process exits.
  *
  *   qbar   device fp32 [B,H,Nq,d]  mean of each query block (as produced by sol_attn_pool)
  *   kc     device fp32 [B,H,Nk,d]  mean of each key block
@@ -203,10 +204,15 @@ sol_status_t sol_attn_read_device_status(sol_stream_t stream);
  *   scale  logit scale, <= 0 selects 1/sqrt(d);  threshold = beta
  *
  * Limit: B*H*d*(d+1) <= sol_attn_thresholds_static_max_floats() (2^20), i.e. B*H <= 63 for d = 128
- * and B*H <= 252 for d = 64; larger problems return SOL_ERR_SCRATCH_LIMIT and launch nothing.
- * The call allocates and frees nothing, enqueues three kernels on `stream` and returns.
- * The first call on each device looks up the array's device address (a runtime query, not an
- * allocation); make that first call outside any stream capture.
+ * and B*H <= 252 for d = 64; larger problems return SOL_ERR_SCRATCH_LIMIT and launch nothing.  A NaN
+ * threshold or a NaN or infinite scale is SOL_ERR_INVALID_ARG, a device that is not compute capability
+ * 10.x SOL_ERR_UNSUPPORTED_ARCH, both before anything is launched.
+ * The FIRST call on each device is a set-up call: it makes the CUDA runtime load the part of the library
+ * that holds the array -- which is when the 4 MiB are reserved on that device and can, like any module
+ * load, fail (SOL_ERR_STATIC_SCRATCH) or synchronise -- and looks up the array's device address.  Make
+ * that first call at start-up, before the process reserves its memory and outside any stream capture.
+ * Every later call allocates and frees nothing, enqueues three kernels on `stream` and returns.  The
+ * address is kept for the life of the process; after a cudaDeviceReset() the library has to be reloaded.
  * All calls on a device share the one array and every call overwrites the part it uses before
  * reading it, so nothing needs clearing between calls -- but two calls that overlap on the GPU
  * (different streams, no ordering) race on it and must be serialised by the caller. */

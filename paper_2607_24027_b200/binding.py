@@ -24,6 +24,7 @@ SOL_ERR_WORKSPACE = -4
 SOL_ERR_CUDA = -5
 SOL_ERR_DEVICE_TIMEOUT = -6
 SOL_ERR_SCRATCH_LIMIT = -7
+SOL_ERR_STATIC_SCRATCH = -8
 
 SOL_MODE_SOL, SOL_MODE_DENSE, SOL_MODE_EXACT_ONLY = 0, 1, 2
 SOL_IMPL_AUTO, SOL_IMPL_TCGEN05, SOL_IMPL_MMA_SYNC = 0, 1, 2

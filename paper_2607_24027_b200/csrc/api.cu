@@ -39,20 +39,14 @@ sol_status_t copy_streams(cudaStream_t* in, cudaStream_t* out) {
   return SOL_OK;
 }
 
-sol_status_t check_arch() {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
-  int major = 0;
-  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SOL_ERR_CUDA;
-  return major == 10 ? SOL_OK : SOL_ERR_UNSUPPORTED_ARCH;
-}
+sol_status_t check_arch() { return sol::check_device_arch(); }
 
 // Shape checks common to every entry point.  `fused` adds the fused kernels' restrictions.
 sol_status_t check_shape(int B, int H, int N, int d, int block_q, int block_k, bool fused) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || block_q <= 0 || block_k <= 0) return SOL_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return SOL_ERR_UNSUPPORTED_SHAPE;
   if (block_q > 1024 || block_k > 1024) return SOL_ERR_UNSUPPORTED_SHAPE;
-  if ((long long)B * H > 0x7fffffLL) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)B * H > 65535LL) return SOL_ERR_UNSUPPORTED_SHAPE;   // (batch, head) pairs index gridDim.y in the pre-attention kernels
   if (sol::ceil_div(N, block_k) > 65535 || sol::ceil_div(N, block_q) > 65535) return SOL_ERR_UNSUPPORTED_SHAPE;
   if ((long long)B * H * sol::ceil_div(N, block_q) > 0x7fffffffLL) return SOL_ERR_UNSUPPORTED_SHAPE;   // work items are counted in int32
   if (fused && (block_q != block_k || (block_q != 64 && block_q != 128))) return SOL_ERR_UNSUPPORTED_SHAPE;
@@ -95,6 +89,17 @@ sol_status_t run_pool(const sol::Problem& p, const void* q, const void* k, const
 
 }  // namespace
 
+namespace sol {
+void count_launches(int n) { g_launches += n; }
+sol_status_t check_device_arch() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SOL_ERR_CUDA;
+  return major == 10 ? SOL_OK : SOL_ERR_UNSUPPORTED_ARCH;
+}
+}  // namespace sol
+
 extern "C" {
 
 const char* sol_attn_status_string(sol_status_t s) {
@@ -107,6 +112,7 @@ const char* sol_attn_status_string(sol_status_t s) {
     case SOL_ERR_CUDA: return "SOL_ERR_CUDA";
     case SOL_ERR_DEVICE_TIMEOUT: return "SOL_ERR_DEVICE_TIMEOUT";
     case SOL_ERR_SCRATCH_LIMIT: return "SOL_ERR_SCRATCH_LIMIT";
+    case SOL_ERR_STATIC_SCRATCH: return "SOL_ERR_STATIC_SCRATCH";
     default: return "SOL_ERR_UNKNOWN";
   }
 }

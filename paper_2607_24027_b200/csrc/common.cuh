@@ -101,6 +101,10 @@ inline WsPtrs make_ptrs(void* base, const WsLayout& w) {
   return p;
 }
 
+// Host-side helpers shared by the files that implement entry points (defined in api.cu).
+void count_launches(int n);            // adds to the library's launch counter (sol_attn_launch_count)
+sol_status_t check_device_arch();      // SOL_OK on compute capability 10.x, else SOL_ERR_UNSUPPORTED_ARCH
+
 // ---- launchers (each returns the cudaError_t of its launches; all work goes to `stream`) ----
 
 // Pooling pre-pass: Qbar, KC, VC (+ bf16 operand copies).  q may be null.

@@ -35,6 +35,8 @@
 //
 // Every mbarrier wait is bounded: when one expires the CTA records SOL_ERR_DEVICE_TIMEOUT in the
 // workspace status word, all roles drain, TMEM is released and the kernel returns.
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "tmap.cuh"
@@ -99,7 +101,8 @@ struct Shared {
   uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
   uint64_t q_full, q_empty;
   uint64_t s_full[2], p_full[2][2], pv_done[2];   // indexed by score buffer (and warpgroup)
-  uint64_t x_full, x_done;      // rendezvous of the two softmax warpgroups at the end of a work item
+  uint64_t x_full;              // rendezvous of the two softmax warpgroups at the end of a work item
+  uint64_t o_free;              // all 8 softmax warps have read both accumulators of the finished work item
   uint64_t kc_full[2];          // router staging buffers filled
   uint64_t mma_drain[2];        // abort path only: all MMAs issued by a role have retired
   uint32_t tmem_base;
@@ -121,6 +124,7 @@ struct Params {
   int rows_inner;               // coordinate order of the q/k/v tensor maps: (c, row, h, b) or (c, h, row, b)
   long long wait_limit;         // SM clocks after which a bounded wait gives up
   int withhold_tile;            // test hook: >= 0: the P V role leaves out the completion signal of this tile
+  int out_aligned32;            // every output row piece starts on a 32-byte boundary (32-byte stores are legal)
 };
 
 template <class S>
@@ -209,6 +213,8 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
   const int n_chunks = ceil_div(p.Nk, kBlk);
   const int mask_words = ceil_div(p.Nk, 32);
   const float inv_sl2 = 1.f / (p.scale * 1.4426950408889634f);   // biases are stored in raw-score units
+  const float bias_full = log2f((float)kBlk) * inv_sl2;                          // log2 n_j of a full block ...
+  const float bias_last = log2f((float)(p.N - (p.Nk - 1) * kBlk)) * inv_sl2;     // ... and of the ragged last one
   bool alive = true;
   PROF_DECL
   if (lane == 0) CTATRACE(0, prof::gtimer());
@@ -299,7 +305,7 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
         const unsigned m = __ballot_sync(full, sel);
         const bool valid = j < p.Nk;
         any_unselected |= (valid && !sel);
-        rec.bias[g * 32 + lane] = (valid && !sel) ? log2f((float)min(kBlk, p.N - j * kBlk)) * inv_sl2 : -INFINITY;
+        rec.bias[g * 32 + lane] = (valid && !sel) ? (j == p.Nk - 1 ? bias_last : bias_full) : -INFINITY;
         if (sel) rec.desc[1 + n_sel + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(j * kBlk) << 5;
         n_sel += __popc(m);
         if (p.mask_out && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
@@ -368,15 +374,20 @@ __device__ void producer_role(Shared<C>& sm, const Params& p, unsigned char* sQ,
   Cursor<C> cur_k, cur_v;
   PROF_DECL
   // pooled = true: KC / mean-V operands, dense [B*H][Nk][d]; else q, k, v in the caller's layout.
-  // A tile is C::kBoxes boxes of 64 channels, each `box_bytes` long in shared memory.
-  auto load_tile = [&](const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row, const Record<C>* rec,
-                       bool pooled, int bytes, int box_bytes) {
-    mbar_arrive_expect_tx(full, bytes);
+  // A tile is C::kBoxes boxes of 64 channels, each kBox bytes long in shared memory.
+  auto load_tile = [&](auto bytes_c, auto box_c, const CUtensorMap* tm, uint64_t* full, unsigned char* dst, int row,
+                       const Record<C>* rec, bool pooled) {
+    constexpr int kBytes = decltype(bytes_c)::value, kBox = decltype(box_c)::value;
+    mbar_arrive_expect_tx(full, kBytes);
     const bool rows_inner = pooled || p.rows_inner;
     const int c1 = rows_inner ? row : rec->h, c2 = rows_inner ? rec->h : row;
-#pragma unroll
-    for (int c = 0; c < C::kBoxes; ++c) tma_load_4d(dst + c * box_bytes, tm, full, 64 * c, c1, c2, rec->b);
+    tma_load_4d(dst, tm, full, 0, c1, c2, rec->b);
+    if constexpr (C::kBoxes == 2) tma_load_4d(dst + kBox, tm, full, 64, c1, c2, rec->b);
   };
+  using QBytes = std::integral_constant<int, C::kQBytes>;
+  using QBox = std::integral_constant<int, C::kQBoxBytes>;
+  using TBytes = std::integral_constant<int, C::kTileBytes>;
+  using TBox = std::integral_constant<int, C::kBoxBytes>;
   auto release = [&](uint32_t r) { mbar_arrive(&sm.rec_empty[r]); };
   bool k_end = false, have_k = false, ok = true;
   uint32_t dk = 0;
@@ -399,7 +410,7 @@ __device__ void producer_role(Shared<C>& sm, const Params& p, unsigned char* sQ,
         const uint32_t par = (n_item & 1) ^ 1;
         if (n_k != n_v && !mbar_try_wait(&sm.q_empty, par)) break;
         if (!WAIT(&sm.q_empty, par, 2)) { ok = false; break; }                  // prof 2: Q slot busy
-        load_tile(tm_q, &sm.q_full, sQ, cur_k.rec->q_row, cur_k.rec, false, C::kQBytes, C::kQBoxBytes);
+        load_tile(QBytes{}, QBox{}, tm_q, &sm.q_full, sQ, cur_k.rec->q_row, cur_k.rec, false);
         ++n_item;
         dk &= ~kTileFirst;
       }
@@ -408,8 +419,8 @@ __device__ void producer_role(Shared<C>& sm, const Params& p, unsigned char* sQ,
       if (!WAIT(&sm.k_empty[s], ((n_k / kKStages) & 1) ^ 1, 1)) { ok = false; break; }   // prof 1: K ring full
       {
         PROF_T0
-        load_tile((dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes, (int)(dk >> 5),
-                  cur_k.rec, (dk & kTileApprox) != 0, kTileBytes, C::kBoxBytes);
+        load_tile(TBytes{}, TBox{}, (dk & kTileApprox) ? tm_kc : tm_k, &sm.k_full[s], sKV + (size_t)s * kTileBytes,
+                  (int)(dk >> 5), cur_k.rec, (dk & kTileApprox) != 0);
         PROF_ADD(4)                                                                    // prof 4: issuing K copies
       }
       ++n_k;
@@ -433,8 +444,8 @@ __device__ void producer_role(Shared<C>& sm, const Params& p, unsigned char* sQ,
     if (!WAIT(&sm.v_empty[s], ((n_v / kVStages) & 1) ^ 1, 3)) { ok = false; break; }     // prof 3: V ring full
     {
       PROF_T0
-      load_tile((dv & kTileApprox) ? tm_vm : tm_v, &sm.v_full[s], sKV + (size_t)(kKStages + s) * kTileBytes,
-                (int)(dv >> 5), cur_v.rec, (dv & kTileApprox) != 0, kTileBytes, C::kBoxBytes);
+      load_tile(TBytes{}, TBox{}, (dv & kTileApprox) ? tm_vm : tm_v, &sm.v_full[s],
+                sKV + (size_t)(kKStages + s) * kTileBytes, (int)(dv >> 5), cur_v.rec, (dv & kTileApprox) != 0);
       PROF_ADD(5)                                                                      // prof 5: issuing V copies
     }
     ++n_v;
@@ -561,7 +572,7 @@ __device__ void mma_pv_role(Shared<C>& sm, const Params& p, unsigned char* sKV, 
   // V is the MN-major operand: its 64-channel boxes are C::kBoxBytes apart (leading offset), groups of
   // 8 key rows 1024 bytes apart; a K-step of 16 keys advances the start by 2048 bytes.
   const uint32_t kv_lo = (smem_addr(sKV + kKStages * kTileBytes) >> 4) | ((uint32_t)(C::kBoxBytes >> 4) << 16);
-  uint32_t g = 0;
+  uint32_t g = 0, n_item = 0;
   uint32_t slot = 0, slot_parity = 0;          // ring position of V(g)
   Cursor<C> cur;
   const bool leader = elect_one();             // warp-uniform role, one issuing lane (see mma_qk_role)
@@ -576,6 +587,10 @@ __device__ void mma_pv_role(Shared<C>& sm, const Params& p, unsigned char* sKV, 
     if (!mbar_wait(&sm.v_full[slot], slot_parity, &sm.abort_flag, wait_limit)) { ok = false; break; }
     const uint32_t v_lo = kv_lo + slot * (kTileBytes >> 4);
     const uint32_t acc_first = (dsc & kTileFirst) ? 0u : 1u;
+    if ((dsc & kTileFirst) && n_item++ > 0) {
+      // the first P V of a work item overwrites O0 / O1: the previous item's merge must have read them
+      if (!mbar_wait(&sm.o_free, (n_item - 2) & 1, &sm.abort_flag, wait_limit)) { ok = false; break; }
+    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (!mbar_wait(&sm.p_full[h][b], (g >> 1) & 1, &sm.abort_flag, wait_limit)) { ok = false; break; }
@@ -637,7 +652,7 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
 #define SWAIT(bar, parity, slot) __all_sync(full, WAIT(bar, parity, slot))
   for (;;) {
     const uint32_t dsc = next_desc(sm, cur, wait_limit, PROF_ACC(0), release);        // prof 0: no record yet
-    if (__any_sync(full, dsc == kDescAbort)) { flag_abort(sm, p, 400); break; }
+    if (dsc == kDescAbort) { flag_abort(sm, p, 400); break; }
     if (dsc == kDescStop) break;
     const bool first = (dsc & kTileFirst) != 0;
 
@@ -647,7 +662,9 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
       const bool approx = (dsc & kTileApprox) != 0;
       const int cols_valid = approx ? kBlk : min(kBlk, p.N - (int)(dsc >> 5));
       const bool general = approx || cols_valid < kBlk;
-      if (!SWAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }  // prof 1: S not ready
+      // (no vote on this wait, the one wait of every tile: the 32 lanes poll the same barrier, abort flag
+      //  and clock in lockstep and leave the loop together; the rarer waits below are made uniform by a vote)
+      if (!WAIT(&sm.s_full[b], (g >> 1) & 1, 1)) { flag_abort(sm, p, 401); break; }   // prof 1: S not ready
       tc_fence_after();
       if (first && warp_in_group == 0 && lane == 0) { ITRACE(n_item, h ? 11 : 5); g_item0 = g; }
       // ---- this group's half row of S (kHalf fp32) into registers with one wait
@@ -783,14 +800,19 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
         tmem_ld_32x32b_x32(t_o + h * kOutCh + c * 32, a);
         tmem_ld_32x32b_x32(t_o_other + h * kOutCh + c * 32, bb);
         tmem_ld_wait();
+        if (c == kOutCh / 32 - 1) {
+          // both accumulators are in registers: the next item's first P V may overwrite them
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.o_free);
+        }
         if (row < q_rows) {
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            uint4 pk;
-            uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
+          for (int x = 0; x < 2; ++x) {                 // 32 bytes (16 channels) per store
+            uint32_t pw[8];
 #pragma unroll
-            for (int y = 0; y < 4; ++y) {
-              const int e0 = x * 8 + 2 * y;
+            for (int y = 0; y < 8; ++y) {
+              const int e0 = x * 16 + 2 * y;
               // a partial accumulator that never received a tile may hold anything: weight 0 must win
               const float v0 = (w_own > 0.f ? __uint_as_float(a[e0]) * c_own : 0.f) +
                                (w_other > 0.f ? __uint_as_float(bb[e0]) * c_other : 0.f);
@@ -799,15 +821,16 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
               __nv_bfloat162 hh = __floats2bfloat162_rn(v0, v1);
               pw[y] = *reinterpret_cast<uint32_t*>(&hh);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = pk;
+            if (p.out_aligned32) {
+              st_global_v8(orow + c * 32 + x * 16, pw);
+            } else {                                    // the interface only asks for 16-byte alignment
+              uint4* dst = reinterpret_cast<uint4*>(orow + c * 32 + x * 16);
+              dst[0] = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+              dst[1] = make_uint4(pw[4], pw[5], pw[6], pw[7]);
+            }
           }
         }
       }
-      tc_fence_before();
-      // neither group may start the next item (whose first P V overwrites O0 / O1) before both
-      // have finished reading
-      mbar_arrive(&sm.x_done);
-      if (!SWAIT(&sm.x_done, n_merge & 1, 6)) { flag_abort(sm, p, 405); break; }
       if (warp_in_group == 0 && lane == 0) ITRACE(n_item, h ? 14 : 9);
       ++n_merge;
     } else if (row < q_rows) {
@@ -848,7 +871,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       mbar_init(&sm.p_full[0][b], 4);
       mbar_init(&sm.p_full[1][b], 4);
     }
-    mbar_init(&sm.x_full, 256); mbar_init(&sm.x_done, 256);
+    mbar_init(&sm.x_full, 256); mbar_init(&sm.o_free, 8);
     mbar_init(&sm.kc_full[0], 1); mbar_init(&sm.kc_full[1], 1);
     mbar_init(&sm.mma_drain[0], 1); mbar_init(&sm.mma_drain[1], 1);
     fence_mbar_init();
@@ -905,6 +928,8 @@ cudaError_t launch_instance(const Problem& p, const __nv_bfloat16* q, const __nv
   prm.mode = p.mode; prm.scale = p.scale; prm.forced = p.forced;
   prm.st = p.st; prm.rows_inner = rows_inner ? 1 : 0;
   prm.wait_limit = g_wait_limit; prm.withhold_tile = g_withhold_tile;
+  prm.out_aligned32 = (reinterpret_cast<uintptr_t>(out) % 32 == 0 && (p.st.row * 2) % 32 == 0 && (p.st.head * 2) % 32 == 0 &&
+                       (p.st.batch * 2) % 32 == 0) ? 1 : 0;
 
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -169,5 +169,6 @@ extern "C" sol_status_t sol_attn_route_materialized(const float* qbar, const flo
   if (cudaFuncSetAttribute(row_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return SOL_ERR_CUDA;
   row_select_kernel<<<dim3(Nq, BH), 256, smem, st>>>(proxy_map, Nq, Nk, npad, policy, param, order, tau, counts);
+  sol::count_launches(2);
   return cudaGetLastError() == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }

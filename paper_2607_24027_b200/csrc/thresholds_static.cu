@@ -7,14 +7,18 @@
 // synchronise the device and stall a latency-critical loop.  The regular entry points keep
 // their intermediate moments in a caller-provided workspace; this one keeps them in a fixed
 // array that lives inside the library image on every GPU that loads it.
+#include <cmath>
 #include <mutex>
 
 #include "common.cuh"
 
 namespace {
 
-// 4 MiB of device memory per GPU, held from the moment the library is loaded until exit.
-// Layout for one call: m_K [BH][d] followed by C_K [BH][d][d].
+// 4 MiB of device memory per GPU.  The array belongs to this file's CUDA module, which the runtime
+// loads on a device the first time something of the module is used there: the first call of the entry
+// point on a device therefore loads the module and reserves the 4 MiB (it can fail, or synchronise, like
+// any module load); from then on the memory is held until the process exits and later calls touch no
+// allocator.  Layout for one call: m_K [BH][d] followed by C_K [BH][d][d].
 constexpr size_t kScratchFloats = size_t(1) << 20;
 static __device__ __align__(256) float g_scratch[kScratchFloats];
 
@@ -23,7 +27,9 @@ std::mutex g_mu;
 float* g_scratch_ptr[kMaxDevices] = {nullptr};   // device address of g_scratch, per device
 
 // `g_scratch` in HOST code is only a handle for the runtime, not a device address; the address a
-// kernel may dereference has to be asked for, once per device, with that device current.
+// kernel may dereference has to be asked for, once per device, with that device current.  The
+// address is cached for the life of the process: a cudaDeviceReset() in between invalidates it, and
+// the library must then be reloaded.
 sol_status_t scratch_for_current_device(float** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
@@ -31,7 +37,10 @@ sol_status_t scratch_for_current_device(float** out) {
   std::lock_guard<std::mutex> lock(g_mu);
   if (!g_scratch_ptr[dev]) {
     float* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_scratch) != cudaSuccess || !p) return SOL_ERR_CUDA;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();                            // leave no sticky-looking error behind
+      return SOL_ERR_STATIC_SCRATCH;
+    }
     g_scratch_ptr[dev] = p;
   }
   *out = g_scratch_ptr[dev];
@@ -83,7 +92,9 @@ __global__ void __launch_bounds__(256) static_key_cov(const float* __restrict__ 
 }
 
 // mu_i = s Qbar_i . m_K, sigma_i = s sqrt(Qbar_i C_K Qbar_i^T), tau_i = mu_i + beta sigma_i.
-// One warp per query block; lane l owns rows l, l+32, ... of C_K.
+// One warp per query block; lane l owns rows l, l+32, ... of C_K (the lanes of a warp read C_K a row
+// apart, i.e. uncoalesced; the matrix is 64 KB per head and stays in cache, and this kernel is a
+// fraction of a percent of a call).
 __global__ void __launch_bounds__(256) static_tau(const float* __restrict__ qbar, const float* __restrict__ mk,
                                                   const float* __restrict__ cov, float* __restrict__ mu,
                                                   float* __restrict__ sigma, float* __restrict__ tau, int Nq, int d,
@@ -122,13 +133,15 @@ extern "C" sol_status_t sol_attn_thresholds_static(const float* qbar, const floa
                                                    float* tau, sol_stream_t stream) {
   if (!qbar || !kc || !mu || !sigma || !tau) return SOL_ERR_INVALID_ARG;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || threshold != threshold) return SOL_ERR_INVALID_ARG;
+  if (scale != scale || isinf(scale)) return SOL_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return SOL_ERR_UNSUPPORTED_SHAPE;
   if (Nq > 65535 * 8 || (long long)B * H > 65535) return SOL_ERR_UNSUPPORTED_SHAPE;
   const size_t bh = (size_t)B * H;
   if (bh * d * ((size_t)d + 1) > kScratchFloats) return SOL_ERR_SCRATCH_LIMIT;
-  float* scratch = nullptr;
-  sol_status_t s = scratch_for_current_device(&scratch);
+  sol_status_t s = sol::check_device_arch();
   if (s != SOL_OK) return s;
+  float* scratch = nullptr;
+  if ((s = scratch_for_current_device(&scratch)) != SOL_OK) return s;
   float* mk = scratch;
   float* cov = scratch + bh * d;
   const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)d);
@@ -136,6 +149,7 @@ extern "C" sol_status_t sol_attn_thresholds_static(const float* qbar, const floa
   static_key_mean<<<(unsigned)bh, d, 0, st>>>(kc, mk, Nk, d);
   static_key_cov<<<dim3(d / 16, (unsigned)bh), 256, 0, st>>>(kc, mk, cov, Nk, d);
   static_tau<<<dim3((Nq + 7) / 8, (unsigned)bh), 256, 0, st>>>(qbar, mk, cov, mu, sigma, tau, Nq, d, sc, threshold);
+  sol::count_launches(3);
   return cudaGetLastError() == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
 

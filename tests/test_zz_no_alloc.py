@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import sol_attn_oracle as orc
 from paper_2607_24027_b200 import synth
 from paper_2607_24027_b200.configs import WORKLOADS, load_betas
 from tests import helpers as hp
@@ -66,6 +67,40 @@ def test_static_thresholds_match_workspace_thresholds_twice():
             assert torch.isinf(tau).all() and torch.isinf(ws.tau).all()
         else:
             _close(tau, ws.tau)
+
+
+def test_static_thresholds_match_the_oracle_and_leave_device_memory_alone():
+    """The same numbers straight against the CPU oracle (row statistics of the proxy map, Eq. 4), and
+    the point of the entry point itself: a call that is not the first one on the device changes nothing
+    in the device's memory accounting (the first call loads the module that holds the array)."""
+    from paper_2607_24027_b200 import binding as sb
+    sb.lib()
+    wl = WORKLOADS["image"]
+    beta = load_betas()["image"][0.3]
+    ws = _reference(sb, wl, beta)
+    qb, kb, vb = synth.generate(wl)
+    _static(sb, ws, beta)                                   # set-up call on this device, if none came before
+    qbar, kc = ws.qbar.contiguous(), ws.kc.contiguous()
+    mu, sigma, tau = (torch.full_like(ws.tau, float("nan")) for _ in range(3))
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    launches_before = sb.sol_attn_launch_count()
+    for _ in range(3):
+        sb.sol_attn_thresholds_static(qbar, kc, beta, mu, sigma, tau)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, (free_before, free_after)
+    assert sb.sol_attn_launch_count() - launches_before == 9   # three kernels per call, all counted
+    for h in (0, wl.heads - 1):
+        r = orc.routing(synth.widen(qb[0, h], np.float64), synth.widen(kb[0, h], np.float64),
+                        synth.widen(vb[0, h], np.float64), wl.block, wl.block, beta)
+        np.testing.assert_allclose(mu[0, h].cpu().numpy(), r.mu, rtol=0, atol=2e-5)
+        np.testing.assert_allclose(sigma[0, h].cpu().numpy(), r.sigma, rtol=1e-4, atol=2e-5)
+        np.testing.assert_allclose(tau[0, h].cpu().numpy(), r.tau, rtol=0, atol=5e-5)
+    # argument checks happen before anything is launched
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_thresholds_static(qbar, kc, beta, mu, sigma, tau, scale=float("inf"))
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
 
 
 def test_static_thresholds_reject_oversized_problems():
