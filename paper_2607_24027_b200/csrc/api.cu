@@ -19,24 +19,44 @@ std::atomic<int64_t> g_launches{0};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Two copy streams per device for the host-buffer entry point, made on first use and kept for the
-// life of the process (streams are host-side objects; no device memory is involved).
+// Two copy streams and four events per device for the host-buffer entry point, made on first use and
+// kept for the life of the process (host-side objects; no device memory is involved).  An event may be
+// recorded again and again: a cudaStreamWaitEvent waits for the record that precedes it.
 constexpr int kMaxDevices = 64;
 std::mutex g_stream_mu;
-cudaStream_t g_copy_in[kMaxDevices] = {nullptr}, g_copy_out[kMaxDevices] = {nullptr};
+struct HostPath {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, copied = nullptr, computed = nullptr, done = nullptr;
+};
+HostPath g_host[kMaxDevices];
 
-sol_status_t copy_streams(cudaStream_t* in, cudaStream_t* out) {
+sol_status_t host_path(HostPath* hp) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SOL_ERR_CUDA;
   if (dev < 0 || dev >= kMaxDevices) return SOL_ERR_UNSUPPORTED_SHAPE;
   std::lock_guard<std::mutex> lock(g_stream_mu);
-  if (!g_copy_in[dev]) {
-    if (cudaStreamCreateWithFlags(&g_copy_in[dev], cudaStreamNonBlocking) != cudaSuccess) return SOL_ERR_CUDA;
-    if (cudaStreamCreateWithFlags(&g_copy_out[dev], cudaStreamNonBlocking) != cudaSuccess) return SOL_ERR_CUDA;
+  HostPath& h = g_host[dev];
+  if (!h.done) {
+    if (cudaStreamCreateWithFlags(&h.in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h.out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.copied, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.computed, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.done, cudaEventDisableTiming) != cudaSuccess)
+      return SOL_ERR_CUDA;
   }
-  *in = g_copy_in[dev];
-  *out = g_copy_out[dev];
+  *hp = h;
   return SOL_OK;
+}
+
+// bytes of one tensor per group of heads on the host path (SOL_ATTN_HOST_GROUP_BYTES may change between calls)
+size_t host_group_bytes() {
+  size_t want = size_t(64) << 20;                            // about 64 MB per tensor and group
+  if (const char* env = getenv("SOL_ATTN_HOST_GROUP_BYTES")) {
+    const long long v = atoll(env);
+    if (v > 0) want = (size_t)v;
+  }
+  return want;
 }
 
 sol_status_t check_arch() { return sol::check_device_arch(); }
@@ -256,48 +276,33 @@ sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* h
   if (!g_bound.ws) return SOL_ERR_WORKSPACE;
   if (g_bound.bytes < sol_attn_workspace_bytes(B, H, N, d, block_q, block_k)) return SOL_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaStream_t s_in = nullptr, s_out = nullptr;
-  if ((s = copy_streams(&s_in, &s_out)) != SOL_OK) return s;
+  HostPath hp;
+  if ((s = host_path(&hp)) != SOL_OK) return s;
 
   // Heads are independent, so the call is cut into groups of heads and pipelined: while the
   // kernels work on one group (on the caller's stream), the next group's q, k, v travel to the
   // device on one copy stream and the previous group's output travels back on another.
   const int BH = B * H, Nq = sol::ceil_div(N, block_q);
   const size_t head_bytes = (size_t)N * d * 2;
-  size_t want = size_t(64) << 20;                            // about 64 MB per tensor and group
-  if (const char* env = getenv("SOL_ATTN_HOST_GROUP_BYTES")) {    // tuning / test knob
-    const long long v = atoll(env);
-    if (v > 0) want = (size_t)v;
-  }
+  const size_t want = host_group_bytes();
   int per = (int)((want + head_bytes - 1) / head_bytes);
   if (per < 1) per = 1;
   if (per > BH) per = BH;
-  auto fail = [](cudaEvent_t a, cudaEvent_t b) {
-    if (a) cudaEventDestroy(a);
-    if (b) cudaEventDestroy(b);
-    return SOL_ERR_CUDA;
-  };
   // copies must not overtake work already queued on the caller's stream (it may still use dq...)
-  cudaEvent_t e0 = nullptr;
-  if (cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
-  if (cudaEventRecord(e0, st) != cudaSuccess || cudaStreamWaitEvent(s_in, e0, 0) != cudaSuccess ||
-      cudaStreamWaitEvent(s_out, e0, 0) != cudaSuccess)
-    return fail(e0, nullptr);
-  cudaEventDestroy(e0);
+  if (cudaEventRecord(hp.start, st) != cudaSuccess || cudaStreamWaitEvent(hp.in, hp.start, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(hp.out, hp.start, 0) != cudaSuccess)
+    return SOL_ERR_CUDA;
   bool first = true;
   for (int h0 = 0; h0 < BH; h0 += per) {
     const int nh = (BH - h0 < per) ? BH - h0 : per;
     const size_t off = (size_t)h0 * head_bytes, bytes = (size_t)nh * head_bytes;
     auto at = [off](const void* p) { return static_cast<const char*>(p) + off; };
     auto at_w = [off](void* p) { return static_cast<char*>(p) + off; };
-    cudaEvent_t e_in = nullptr, e_done = nullptr;
-    if (cudaEventCreateWithFlags(&e_in, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
-    if (cudaEventCreateWithFlags(&e_done, cudaEventDisableTiming) != cudaSuccess) return fail(e_in, nullptr);
-    if (cudaMemcpyAsync(at_w(dq), at(hq), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
-        cudaMemcpyAsync(at_w(dk), at(hk), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
-        cudaMemcpyAsync(at_w(dv), at(hv), bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
-        cudaEventRecord(e_in, s_in) != cudaSuccess || cudaStreamWaitEvent(st, e_in, 0) != cudaSuccess)
-      return fail(e_in, e_done);
+    if (cudaMemcpyAsync(at_w(dq), at(hq), bytes, cudaMemcpyHostToDevice, hp.in) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(dk), at(hk), bytes, cudaMemcpyHostToDevice, hp.in) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(dv), at(hv), bytes, cudaMemcpyHostToDevice, hp.in) != cudaSuccess ||
+        cudaEventRecord(hp.copied, hp.in) != cudaSuccess || cudaStreamWaitEvent(st, hp.copied, 0) != cudaSuccess)
+      return SOL_ERR_CUDA;
     sol_attn_args a{};
     a.q = at_w(dq); a.k = at_w(dk); a.v = at_w(dv); a.out = at_w(dout);
     a.B = 1; a.H = nh; a.N = N; a.d = d; a.block_q = block_q; a.block_k = block_k;
@@ -307,18 +312,14 @@ sol_status_t sol_attn_forward_host(const void* hq, const void* hk, const void* h
     a.stream = stream;
     s = forward_impl(&a, !first);
     first = false;
-    if (s != SOL_OK) { fail(e_in, e_done); return s; }
-    if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(s_out, e_done, 0) != cudaSuccess ||
-        cudaMemcpyAsync(at_w(hout), at(dout), bytes, cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
-      return fail(e_in, e_done);
-    cudaEventDestroy(e_in);
-    cudaEventDestroy(e_done);
+    if (s != SOL_OK) return s;
+    if (cudaEventRecord(hp.computed, st) != cudaSuccess || cudaStreamWaitEvent(hp.out, hp.computed, 0) != cudaSuccess ||
+        cudaMemcpyAsync(at_w(hout), at(dout), bytes, cudaMemcpyDeviceToHost, hp.out) != cudaSuccess)
+      return SOL_ERR_CUDA;
   }
   // the caller's stream ends where the last copy back ends
-  cudaEvent_t e1 = nullptr;
-  if (cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess) return SOL_ERR_CUDA;
-  if (cudaEventRecord(e1, s_out) != cudaSuccess || cudaStreamWaitEvent(st, e1, 0) != cudaSuccess) return fail(e1, nullptr);
-  cudaEventDestroy(e1);
+  if (cudaEventRecord(hp.done, hp.out) != cudaSuccess || cudaStreamWaitEvent(st, hp.done, 0) != cudaSuccess)
+    return SOL_ERR_CUDA;
   return SOL_OK;
 }
 

@@ -147,10 +147,9 @@ def test_p4_exhaustive_tiny(L, d, b):
     _, kc, vc, _ = orc.pool(q, k, v, b, b)
     scale = 0.5
     rows = list(itertools.product([False, True], repeat=nb))
-    step = 1 if len(rows) <= 16 else 5          # every row pattern when few, a stride else
-    for a, pat in enumerate(rows[::step]):
-        # every query block gets a (different) pattern; all patterns are visited
-        mask = np.array([rows[(a * step + 3 * i) % len(rows)] for i in range(nb)])
+    for a in range(len(rows)):
+        # every query block gets a (different) pattern; each block sees every one of the 2^nb patterns
+        mask = np.array([rows[(a + 3 * i) % len(rows)] for i in range(nb)])
         out, m2 = orc.sol_attn_streaming(q, k, v, kc, vc, None, b, b, chunk=2, scale=scale,
                                          mask_override=mask)
         assert np.array_equal(m2, mask)
