@@ -14,9 +14,12 @@
 
 using namespace sol::ptx;
 
-// mode bit 0: copy stream on; bit 1: score MMAs take A from TMEM; bit 2: no MMAs at all
-__global__ void __launch_bounds__(128) probe_mma(long long* out, const unsigned char* gsrc, int mode, int iters,
-                                                 int src_bytes) {
+// MODE bit 0: copy stream on; bit 1: score MMAs take A from TMEM; bit 2: no MMAs at all;
+// bit 3: score MMAs TMEM x shared in two halves of 64 key columns.
+// The issuing thread's own instructions must not be what is measured: the mode is a template
+// parameter and every descriptor is built before the timed loop.
+template <int MODE>
+__global__ void __launch_bounds__(128) probe_mma(long long* out, const unsigned char* gsrc, int iters, int src_bytes) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* base = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
   __shared__ uint64_t bar, tbar[2];
@@ -36,30 +39,47 @@ __global__ void __launch_bounds__(128) probe_mma(long long* out, const unsigned 
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
   const unsigned char* src = gsrc + (size_t)blockIdx.x * src_bytes;
-  if (threadIdx.x == 0 && !(mode & 4)) {
+  if (threadIdx.x == 0 && !(MODE & 4)) {
     const uint32_t a_addr = smem_addr(base), b_addr = smem_addr(base + 32768);
     const uint32_t id_qk = make_idesc_bf16(128, 128, false, false);
+    const uint32_t id_qk64 = make_idesc_bf16(128, 64, false, false);
     const uint32_t id_pv = make_idesc_bf16(128, 128, false, true);
-    const long long t0 = clock64();
-    for (int it = 0; it < iters; ++it) {
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint32_t off = (ks / 4) * 16384 + (ks % 4) * 32;
-        if (mode & 2)
-          mma_ts(tmem + (it & 1) * 128, tmem + 256 + ks * 8, make_smem_desc_sw128(b_addr + off, 16, 1024), id_qk, ks > 0);
-        else
-          mma_ss(tmem + (it & 1) * 128, make_smem_desc_sw128(a_addr + off, 16, 1024),
-                 make_smem_desc_sw128(b_addr + off, 16, 1024), id_qk, ks > 0);
-      }
-      for (int ks = 0; ks < 8; ++ks)
-        mma_ts(tmem + 256 + (ks / 4) * 128, tmem + ((it + 1) & 1) * 128 + ks * 8,
-               make_smem_desc_sw128(b_addr + 32768 + ks * 2048, 16384, 1024), id_pv, 1);
+    uint64_t da[8], db[8], db2[8], dv[8];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      const uint32_t off = (ks / 4) * 16384 + (ks % 4) * 32;
+      da[ks] = make_smem_desc_sw128(a_addr + off, 16, 1024);
+      db[ks] = make_smem_desc_sw128(b_addr + off, 16, 1024);
+      db2[ks] = make_smem_desc_sw128(b_addr + off + 8192, 16, 1024);
+      dv[ks] = make_smem_desc_sw128(b_addr + 32768 + ks * 2048, 16384, 1024);
     }
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (int it = 0; it < iters; it += 2) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {               // two tiles per trip: the accumulator choice is static
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          if (MODE & 8) {
+            mma_ts(tmem + u * 128, tmem + 256 + ks * 8, db[ks], id_qk64, ks > 0);
+            mma_ts(tmem + u * 128 + 64, tmem + 256 + ks * 8, db2[ks], id_qk64, ks > 0);
+          } else if (MODE & 2) {
+            mma_ts(tmem + u * 128, tmem + 256 + ks * 8, db[ks], id_qk, ks > 0);
+          } else {
+            mma_ss(tmem + u * 128, da[ks], db[ks], id_qk, ks > 0);
+          }
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) mma_ts(tmem + 256 + (ks / 4) * 128, tmem + (1 - u) * 128 + ks * 8, dv[ks], id_pv, 1);
+      }
+    }
+    const long long t1 = clock64();
     mma_commit(&bar);
     const bool ok = mbar_wait(&bar, 0, &abort_flag);
     out[blockIdx.x * 4 + 0] = clock64() - t0;
-    out[blockIdx.x * 4 + 2] = ok;
+    out[blockIdx.x * 4 + 2] = ok ? (t1 - t0) : -1;      // issue time alone (the loop), or -1 on a timeout
   }
-  if (threadIdx.x == 32 && (mode & 1)) {
+  if (threadIdx.x == 32 && (MODE & 1)) {
     const long long t0 = clock64();
     bool ok = true;
     for (int it = 0; it < iters && ok; ++it) {
@@ -81,12 +101,27 @@ __global__ void __launch_bounds__(128) probe_mma(long long* out, const unsigned 
   if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-// out_dev: int64[4 * grid] = per CTA {MMA cycles, copy cycles, MMA ok, copy ok}; src: grid * src_bytes bytes
-extern "C" int run_probe_mma(long long* out_dev, const unsigned char* src, int mode, int iters, int grid, int src_bytes) {
+template <int MODE>
+static int launch(long long* out_dev, const unsigned char* src, int iters, int grid, int src_bytes) {
   const size_t smem = 160 * 1024 + 1024;
-  if (cudaFuncSetAttribute(probe_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -1;
-  probe_mma<<<grid, 128, smem>>>(out_dev, src, mode, iters, src_bytes);
+  if (cudaFuncSetAttribute(probe_mma<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -1;
+  probe_mma<MODE><<<grid, 128, smem>>>(out_dev, src, iters, src_bytes);
   const cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { printf("cuda error %s\n", cudaGetErrorString(e)); return -2; }
   return 0;
+}
+
+// out_dev: int64[4 * grid] = per CTA {MMA cycles, copy cycles, MMA issue cycles, copy ok}; src: grid * src_bytes bytes;
+// iters must be even
+extern "C" int run_probe_mma(long long* out_dev, const unsigned char* src, int mode, int iters, int grid, int src_bytes) {
+  switch (mode) {
+    case 0: return launch<0>(out_dev, src, iters, grid, src_bytes);
+    case 1: return launch<1>(out_dev, src, iters, grid, src_bytes);
+    case 2: return launch<2>(out_dev, src, iters, grid, src_bytes);
+    case 3: return launch<3>(out_dev, src, iters, grid, src_bytes);
+    case 5: return launch<5>(out_dev, src, iters, grid, src_bytes);
+    case 8: return launch<8>(out_dev, src, iters, grid, src_bytes);
+    case 9: return launch<9>(out_dev, src, iters, grid, src_bytes);
+    default: return -3;
+  }
 }

@@ -37,17 +37,18 @@ def main():
     out = torch.zeros(sms * 4, dtype=torch.int64, device="cuda")
     src = torch.zeros(sms * src_bytes, dtype=torch.uint8, device="cuda")
     names = {0: "scores shared x shared, values TMEM x shared", 1: "  + 64 KB/tile of bulk copies",
-             2: "scores TMEM x shared, values TMEM x shared", 3: "  + 64 KB/tile of bulk copies", 5: "bulk copies alone"}
+             2: "scores TMEM x shared, values TMEM x shared", 3: "  + 64 KB/tile of bulk copies",
+             8: "scores TMEM x shared in two 64-column halves", 9: "  + 64 KB/tile of bulk copies", 5: "bulk copies alone"}
     iters = 512
     for grid in (1, sms):
-        for mode in (0, 1, 2, 3, 5):
+        for mode in (0, 1, 2, 3, 8, 9, 5):
             for _ in range(2):
                 out.zero_()
                 if lib.run_probe_mma(out.data_ptr(), src.data_ptr(), mode, iters, grid, src_bytes) != 0:
                     raise SystemExit("probe failed")
             o = out.view(sms, 4)[:grid].float()
-            print(f"{grid:3d} CTA(s)  {names[mode]:48s} MMAs {o[:, 0].mean().item() / iters:7.1f} cycles/tile   "
-                  f"copies {o[:, 1].mean().item() / iters:7.1f} cycles/tile")
+            print(f"{grid:3d} CTA(s)  {names[mode]:48s} MMAs {o[:, 0].mean().item() / iters:7.1f} cycles/tile "
+                  f"(issue alone {o[:, 2].mean().item() / iters:7.1f})   copies {o[:, 1].mean().item() / iters:7.1f} cycles/tile")
 
 
 if __name__ == "__main__":
