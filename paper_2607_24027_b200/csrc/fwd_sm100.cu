@@ -650,10 +650,22 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
   // A wait that gives up must give up for the whole warp: the loop holds warp-synchronising
   // operations (TMEM loads and stores, votes), so the lanes leave together or not at all.
 #define SWAIT(bar, parity, slot) __all_sync(full, WAIT(bar, parity, slot))
+  // The next descriptor of the open record is read from shared memory while the current tile is being
+  // worked on, so that the read's latency is off the path from one tile to the next.
+  bool peeked = false;
+  uint32_t dsc_peek = 0;
   for (;;) {
-    const uint32_t dsc = next_desc(sm, cur, wait_limit, PROF_ACC(0), release);        // prof 0: no record yet
-    if (dsc == kDescAbort) { flag_abort(sm, p, 400); break; }
-    if (dsc == kDescStop) break;
+    uint32_t dsc;
+    if (peeked) {
+      dsc = dsc_peek;
+      ++cur.e;
+    } else {
+      dsc = next_desc(sm, cur, wait_limit, PROF_ACC(0), release);                     // prof 0: no record yet
+      if (dsc == kDescAbort) { flag_abort(sm, p, 400); break; }
+      if (dsc == kDescStop) break;
+    }
+    peeked = cur.e < cur.end;
+    if (peeked) dsc_peek = cur.rec->desc[cur.e];
     const bool first = (dsc & kTileFirst) != 0;
 
     if (!(dsc & kTileEnd)) {
