@@ -146,3 +146,12 @@ def test_replica_sharding_over_gloo(tmp_path):
     res = json.loads(line)
     assert res["world"] == 2 and res["ms"] == 11.0
     assert res["digests"][0] != res["digests"][1], "ranks must draw different replicas"
+
+
+def test_microbenchmarks_build_and_export_their_entry_points():
+    """The tensor-core and softmax / hand-over probes cross-compile for sm_100a and load without a GPU."""
+    from paper_2607_24027_b200 import mma_probe, softmax_probe
+    mma = ctypes.CDLL(mma_probe.build())
+    assert hasattr(mma, "run_probe_mma")
+    soft = ctypes.CDLL(softmax_probe.build())
+    assert hasattr(soft, "run_probe_softmax") and hasattr(soft, "run_probe_handover")
