@@ -460,7 +460,7 @@ def main():
     line = {
         "metric": METRIC, "value": job_flops / (ms_step * 1e-3) / 1e12, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak" if (args.replicas or world == 1) else "strong",
+        "higher_is_better": True, "scaling": "weak" if args.replicas else "strong",
         "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"{wl.name} density {args.density}", "B": B, "H": H, "N": N, "d": d,
