@@ -337,6 +337,12 @@ def main():
     def kernel_only(b=beta):
         sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl, skip_pool=True)
 
+    mask_buf = torch.zeros(B, H, wl.n_blocks, sb.mask_words(wl.n_blocks), dtype=torch.int32, device="cuda")
+
+    def prepass_step(b=beta, skip_pool=False):   # Eq. (4) decided by the pre-pass kernel, one bit per block pair
+        sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl, skip_pool=skip_pool,
+                               routing=sb.SOL_ROUTING_PREPASS, mask_out=mask_buf)
+
     def dense_step():
         sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, mode=sb.SOL_MODE_DENSE, impl=impl)
 
@@ -396,11 +402,19 @@ def main():
             ms_k = timed(lambda: kernel_only(b), max(3, args.steps // 2), 1)
             dens = cs / float(B * H * wl.n_blocks * wl.n_blocks)
             cf = computed_flops(wl, cs, n_bh=B * H)
-            sweep.append({"mode": "sol", "target_density": rho, "beta": b, "density": dens,
-                          "ms_per_call": ms_f, "kernel_ms": ms_k, "dense_equiv_tflops": dflops / ms_f / 1e9,
-                          "computed_tflops": cf / ms_k / 1e9,
-                          "frac_of_peak_computed": cf / ms_k / 1e9 / peaks["bf16_burst"],
-                          "speedup_vs_dense": ms_dense / ms_f, "one_over_density": 1.0 / dens})
+            entry = {"mode": "sol", "target_density": rho, "beta": b, "density": dens,
+                     "ms_per_call": ms_f, "kernel_ms": ms_k, "dense_equiv_tflops": dflops / ms_f / 1e9,
+                     "computed_tflops": cf / ms_k / 1e9,
+                     "frac_of_peak_computed": cf / ms_k / 1e9 / peaks["bf16_burst"],
+                     "speedup_vs_dense": ms_dense / ms_f, "one_over_density": 1.0 / dens}
+            if impl != sb.SOL_IMPL_MMA_SYNC:
+                # the optional routing pre-pass (SOL_ROUTING_PREPASS): whole call, and mask kernel + fused kernel
+                ms_pf = timed(lambda: prepass_step(b), max(3, args.steps // 2), 1)
+                ms_pk = timed(lambda: prepass_step(b, True), max(3, args.steps // 2), 1)
+                entry["routing_prepass"] = {"ms_per_call": ms_pf, "mask_and_fused_kernel_ms": ms_pk,
+                                            "frac_of_peak_computed": cf / ms_pk / 1e9 / peaks["bf16_burst"],
+                                            "speedup_vs_dense": ms_dense / ms_pf}
+            sweep.append(entry)
         check_status()
 
     # ---- routing latency: the thresholds of Eq. (4)/(5) (what the method needs before its single

@@ -81,6 +81,21 @@ enum {
                              is needed before or after the operator                              */
 };
 
+/* where the comparison of Eq. (4), s_ij > tau_i, is evaluated */
+enum {
+  SOL_ROUTING_FUSED   = 0,  /* inside the fused kernel, as Algorithm 1 has it: no routing decision ever
+                               reaches memory (the default)                                          */
+  SOL_ROUTING_PREPASS = 1   /* by a small kernel before the fused one, kept as ONE BIT per (query block,
+                               key block) pair in `mask_out` (which must then be given; 1.7 MB at
+                               75 600 tokens x 40 heads) and read back by the fused kernel.  The proxy
+                               scores themselves are still never stored.  Same decisions up to fp32
+                               summation order, i.e. identical outside the rounding band of the
+                               threshold.  Pays off at low routing densities, where the in-kernel
+                               router paces the work item; tcgen05 implementation only (with
+                               SOL_IMPL_MMA_SYNC the call returns SOL_ERR_INVALID_ARG); ignored in
+                               SOL_MODE_DENSE                                                         */
+};
+
 /* Human-readable name of a status code; never NULL, static storage. */
 const char* sol_attn_status_string(sol_status_t status);
 
@@ -154,7 +169,9 @@ typedef struct {
   uint32_t* mask_out;                           /* debug: device bitmask [B,H,Nq,ceil(Nk/32)],
                                                    bit j%32 of word j/32 set when block j is in
                                                    S_i; NULL in production (the proxy map is
-                                                   never written to memory otherwise)           */
+                                                   never written to memory otherwise); with
+                                                   SOL_ROUTING_PREPASS: required, written by the
+                                                   pre-pass and read by the fused kernel        */
   sol_stream_t stream;
   int32_t estimator;                            /* SOL_EST_* (0 = Eq. 5 moments)                */
   const uint8_t* forced_blocks;                 /* device uint8 [ceil(N/block_k)] or NULL: key
@@ -164,6 +181,7 @@ typedef struct {
                                                    the paper's MMDiT integrations); shared by all
                                                    batches and heads; counts include them         */
   int32_t layout;                               /* SOL_LAYOUT_* of q, k, v and out (0 = [B,H,N,d]) */
+  int32_t routing;                              /* SOL_ROUTING_* (0 = inside the fused kernel)   */
 } sol_attn_args;
 /* Everything sol_attn_forward_ex enqueues is ordinary work on `stream` (a memset of the status words
  * and kernels), so the call may be captured into a CUDA graph and replayed; sol_attn_forward_host may

@@ -30,6 +30,7 @@ SOL_MODE_SOL, SOL_MODE_DENSE, SOL_MODE_EXACT_ONLY = 0, 1, 2
 SOL_IMPL_AUTO, SOL_IMPL_TCGEN05, SOL_IMPL_MMA_SYNC = 0, 1, 2
 SOL_EST_MOMENTS, SOL_EST_DIAGONAL = 0, 1
 SOL_LAYOUT_BHND, SOL_LAYOUT_BNHD = 0, 1
+SOL_ROUTING_FUSED, SOL_ROUTING_PREPASS = 0, 1
 SOL_ROUTE_TOPK, SOL_ROUTE_TOPP = 0, 1
 
 EXPORTS = [
@@ -65,7 +66,7 @@ class _Args(ctypes.Structure):
         ("counts", ctypes.c_void_p), ("mask_out", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
         ("estimator", ctypes.c_int32), ("forced_blocks", ctypes.c_void_p),
-        ("layout", ctypes.c_int32),
+        ("layout", ctypes.c_int32), ("routing", ctypes.c_int32),
     ]
 
 
@@ -236,7 +237,7 @@ def sol_attn_dense(q, k, v, out, stream=None):
 def sol_attn_forward_ex(q, k, v, out, ws: Workspace, block_q, block_k, threshold=0.0, scale=0.0,
                         mode=SOL_MODE_SOL, impl=SOL_IMPL_AUTO, skip_pool=False, tau_override=None,
                         counts=None, mask_out=None, stream=None, estimator=SOL_EST_MOMENTS, forced_blocks=None,
-                        layout=SOL_LAYOUT_BHND):
+                        layout=SOL_LAYOUT_BHND, routing=SOL_ROUTING_FUSED):
     """``layout=SOL_LAYOUT_BNHD``: q, k, v and out are [B, N, H, d] tensors (heads interleaved)."""
     B, H, N, d = _dims(q)
     if layout == SOL_LAYOUT_BNHD:
@@ -247,7 +248,7 @@ def sol_attn_forward_ex(q, k, v, out, ws: Workspace, block_q, block_k, threshold
               workspace=ws.buf.data_ptr(), workspace_bytes=ws.buf.numel(),
               counts=_ptr(counts if counts is not None else ws.counts), mask_out=_ptr(mask_out),
               stream=_stream(stream), estimator=int(estimator), forced_blocks=_ptr(forced_blocks),
-              layout=int(layout))
+              layout=int(layout), routing=int(routing))
     _check(lib().sol_attn_forward_ex(ctypes.byref(a)), "sol_attn_forward_ex")
 
 

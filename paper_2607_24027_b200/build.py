@@ -14,7 +14,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsol_attn.so")
-SOURCES = ["api.cu", "pool.cu", "fwd_mma_sync.cu", "fwd_sm100.cu", "thresholds_static.cu", "route_materialized.cu"]
+SOURCES = ["api.cu", "pool.cu", "fwd_mma_sync.cu", "fwd_sm100.cu", "thresholds_static.cu", "route_materialized.cu",
+           "route_prepass.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "ptx_sm100.cuh"), os.path.join(CSRC, "tmap.cuh"),
            os.path.join(CSRC, "fwd_sm100_prof.cuh"),
            os.path.join(ROOT, "include", "sol_attn.h")]

@@ -205,16 +205,22 @@ static sol_status_t forward_impl(const sol_attn_args* a, bool keep_status) {
   if (std::isnan(a->scale) || std::isinf(a->scale)) return SOL_ERR_INVALID_ARG;
   if (a->estimator != SOL_EST_MOMENTS && a->estimator != SOL_EST_DIAGONAL) return SOL_ERR_INVALID_ARG;
   if (a->layout != SOL_LAYOUT_BHND && a->layout != SOL_LAYOUT_BNHD) return SOL_ERR_INVALID_ARG;
+  if (a->routing != SOL_ROUTING_FUSED && a->routing != SOL_ROUTING_PREPASS) return SOL_ERR_INVALID_ARG;
+  // the pre-pass keeps its decisions in the caller's mask buffer
+  const bool prepass = a->routing == SOL_ROUTING_PREPASS && a->mode != SOL_MODE_DENSE;
+  if (prepass && !a->mask_out) return SOL_ERR_INVALID_ARG;
   if (!a->workspace || (reinterpret_cast<uintptr_t>(a->workspace) & 1023u) != 0) return SOL_ERR_WORKSPACE;
   if (a->workspace_bytes < sol_attn_workspace_bytes(a->B, a->H, a->N, a->d, a->block_q, a->block_k))
     return SOL_ERR_WORKSPACE;
   if ((s = check_arch()) != SOL_OK) return s;
 
-  const sol::Problem p = make_problem(a->B, a->H, a->N, a->d, a->block_q, a->block_k, a->threshold, a->scale, a->mode,
-                                      a->estimator, a->mode == SOL_MODE_DENSE ? nullptr : a->forced_blocks, a->layout);
+  sol::Problem p = make_problem(a->B, a->H, a->N, a->d, a->block_q, a->block_k, a->threshold, a->scale, a->mode,
+                                a->estimator, a->mode == SOL_MODE_DENSE ? nullptr : a->forced_blocks, a->layout);
+  p.routing = prepass ? SOL_ROUTING_PREPASS : SOL_ROUTING_FUSED;
   int impl = a->impl;
   if (impl == SOL_IMPL_AUTO) impl = sol::fwd_sm100_supports(p) ? SOL_IMPL_TCGEN05 : SOL_IMPL_MMA_SYNC;
   if (impl == SOL_IMPL_TCGEN05 && !sol::fwd_sm100_supports(p)) return SOL_ERR_UNSUPPORTED_SHAPE;
+  if (prepass && impl != SOL_IMPL_TCGEN05) return SOL_ERR_INVALID_ARG;   // only the tcgen05 kernel reads the bits
 
   cudaStream_t stream = static_cast<cudaStream_t>(a->stream);
   const sol::WsLayout lay = sol::make_layout(p.BH, p.Nq, p.Nk, p.d);
@@ -230,6 +236,10 @@ static sol_status_t forward_impl(const sol_attn_args* a, bool keep_status) {
   const float* tau = a->tau_override ? a->tau_override : ws.tau;
   int n = 0;
   cudaError_t e;
+  if (prepass) {
+    e = sol::launch_route_prepass(p, ws, tau, a->mask_out, stream, &n);
+    if (e != cudaSuccess) { g_launches += n; return SOL_ERR_CUDA; }
+  }
   const auto* q = static_cast<const __nv_bfloat16*>(a->q);
   const auto* k = static_cast<const __nv_bfloat16*>(a->k);
   const auto* v = static_cast<const __nv_bfloat16*>(a->v);

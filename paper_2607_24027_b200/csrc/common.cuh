@@ -41,6 +41,7 @@ struct Problem {
   int estimator;     // SOL_EST_*: how sigma_i is obtained
   const uint8_t* forced;   // device [Nk] or null: key blocks that always go to the exact branch
   Strides st;              // SOL_LAYOUT_*: strides of q, k, v, out
+  int routing;             // SOL_ROUTING_*: where the comparison of Eq. (4) is evaluated
 };
 
 // Byte offsets into the workspace (all multiples of 1024).
@@ -113,6 +114,10 @@ cudaError_t launch_pool(const Problem& p, const __nv_bfloat16* q, const __nv_bfl
 
 // Pooled-key moments (Eq. 5) and per-query-block mu, sigma, tau (Eq. 4).
 cudaError_t launch_thresholds(const Problem& p, const WsPtrs& ws, cudaStream_t stream, int* n_launches);
+
+// Routing pre-pass (SOL_ROUTING_PREPASS): one decision bit per (query block, key block) into `mask`.
+cudaError_t launch_route_prepass(const Problem& p, const WsPtrs& ws, const float* tau, uint32_t* mask,
+                                 cudaStream_t stream, int* n_launches);
 
 // Fused forward, warp-level mma.sync implementation (all supported shapes).
 cudaError_t launch_fwd_mma_sync(const Problem& p, const __nv_bfloat16* q, const __nv_bfloat16* k,

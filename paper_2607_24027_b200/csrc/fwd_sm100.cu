@@ -203,7 +203,9 @@ __device__ __forceinline__ uint32_t next_desc(Shared<C>& sm, Cursor<C>& c, long 
 
 // ------------------------------------------------------------------------------------------------
 // router: one warp
-template <class C>
+// kFromMask: the decisions were taken by the routing pre-pass and are read back from the mask (one bit per
+// (query block, key block)) instead of being scored here.
+template <class C, bool kFromMask>
 __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
   constexpr int kD = C::kD, kBlk = C::kBlk, kPieces = C::kD / 4;   // 16-byte pieces per pooled key
   const unsigned full = 0xffffffffu;
@@ -213,6 +215,7 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
   const int n_chunks = ceil_div(p.Nk, kBlk);
   const int mask_words = ceil_div(p.Nk, 32);
   const float inv_sl2 = 1.f / (p.scale * 1.4426950408889634f);   // biases are stored in raw-score units
+  constexpr bool from_mask = kFromMask;
   const float bias_full = log2f((float)kBlk) * inv_sl2;                          // log2 n_j of a full block ...
   const float bias_last = log2f((float)(p.N - (p.Nk - 1) * kBlk)) * inv_sl2;     // ... and of the ragged last one
   bool alive = true;
@@ -227,7 +230,7 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
     const int bh = w / p.Nq, i = w - bh * p.Nq;
     // the pooled query of this work item goes to shared memory (one 16-byte piece per lane)
     float tau_i = 0.f;
-    if (p.mode != SOL_MODE_DENSE) {
+    if (p.mode != SOL_MODE_DENSE && !from_mask) {
       __syncwarp();
       if (lane < kPieces)
         reinterpret_cast<float4*>(sm.qbar_s)[lane] =
@@ -241,7 +244,7 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
     // Bulk-copy one group of 32 pooled keys (contiguous in memory) into a staging buffer;
     // the copy of group n+1 is in flight while group n is scored.
     auto stage_group = [&](int jb) {
-      if (p.mode == SOL_MODE_DENSE || jb >= p.Nk) return;
+      if (p.mode == SOL_MODE_DENSE || from_mask || jb >= p.Nk) return;
       __syncwarp();                                  // every lane is done reading this buffer
       if (lane == 0) {
         const uint32_t buf = n_copy & 1;
@@ -270,6 +273,8 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
         const int j = jbase + lane;
         if (p.mode == SOL_MODE_DENSE) {
           sel = j < p.Nk;
+        } else if (from_mask) {
+          sel = (j < p.Nk) && ((p.mask_out[(size_t)w * mask_words + jbase / 32] >> lane) & 1u);
         } else {
           // lane l scores pooled key jbase + l against the staged rows.  Lane l starts at 16-byte
           // piece l of its row and of the query and walks round, so that the lanes spread over the
@@ -308,7 +313,7 @@ __device__ void router_role(Shared<C>& sm, const Params& p, int lane) {
         rec.bias[g * 32 + lane] = (valid && !sel) ? (j == p.Nk - 1 ? bias_last : bias_full) : -INFINITY;
         if (sel) rec.desc[1 + n_sel + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(j * kBlk) << 5;
         n_sel += __popc(m);
-        if (p.mask_out && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
+        if (p.mask_out && !from_mask && lane == 0 && jbase < p.Nk) p.mask_out[(size_t)w * mask_words + jbase / 32] = m;
       }
       if (!alive) break;
       any_unselected = __any_sync(full, any_unselected);
@@ -858,7 +863,7 @@ __device__ void softmax_role(Shared<C>& sm, const Params& p, uint32_t tmem, int 
   if (lane == 0 && warp_in_group == 0 && h == 0) { PROF_FLUSH(3); CTATRACE(3, prof::gtimer()); }
 }
 
-template <class C>
+template <class C, bool kFromMask>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kc,
@@ -901,7 +906,7 @@ fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (warp < 8) {
     softmax_role<C>(sm, p, tmem, warp / 4, warp % 4, lane);
   } else if (warp == kWarpRouter) {
-    router_role<C>(sm, p, lane);
+    router_role<C, kFromMask>(sm, p, lane);
   } else if (warp == kWarpProducer) {
     if (lane == 0) producer_role<C>(sm, p, sQ, sKV, &tm_q, &tm_k, &tm_v, &tm_kc, &tm_vm);
   } else if (warp == kWarpQK) {
@@ -949,10 +954,17 @@ cudaError_t launch_instance(const Problem& p, const __nv_bfloat16* q, const __nv
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   const size_t smem = 1024 + C::kQBytes + (kKStages + kVStages) * C::kTileBytes + sizeof(Shared<C>);
-  e = cudaFuncSetAttribute(fwd_sm100_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   const int grid = prm.total_work < sms ? prm.total_work : sms;
-  fwd_sm100_kernel<C><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
+  // the pre-pass variant is a kernel of its own, so that the in-kernel router's code is what it is without it
+  if (p.routing == SOL_ROUTING_PREPASS && p.mode != SOL_MODE_DENSE) {
+    e = cudaFuncSetAttribute(fwd_sm100_kernel<C, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    fwd_sm100_kernel<C, true><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
+  } else {
+    e = cudaFuncSetAttribute(fwd_sm100_kernel<C, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    fwd_sm100_kernel<C, false><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvm, prm);
+  }
   if (n_launches) *n_launches += 1;
   return cudaGetLastError();
 }

@@ -97,7 +97,7 @@ def unpack_mask(words: torch.Tensor, n_k: int) -> np.ndarray:
 
 
 def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, scale=0.0, want_mask=True,
-            tau_override=None, ws=None, estimator=0, forced=None, layout=0, skip_pool=False):
+            tau_override=None, ws=None, estimator=0, forced=None, layout=0, skip_pool=False, routing=0):
     """Run the fused forward through the C ABI; returns (out, counts, mask or None, ws).
 
     layout = SOL_LAYOUT_BNHD: q, k, v (and the returned out) are [B, N, H, d].
@@ -114,7 +114,7 @@ def run_gpu(q, k, v, block, beta, mode=sb.SOL_MODE_SOL, impl=sb.SOL_IMPL_AUTO, s
         mask_words = torch.zeros(B, H, ws.view.n_q_blocks, sb.mask_words(nk), dtype=torch.int32, device="cuda")
     sb.sol_attn_forward_ex(q, k, v, out, ws, block, block, threshold=beta, scale=scale, mode=mode, impl=impl,
                            mask_out=mask_words, tau_override=tau_override, estimator=estimator, layout=layout,
-                           skip_pool=skip_pool,
+                           skip_pool=skip_pool, routing=routing,
                            forced_blocks=(None if forced is None else torch.from_numpy(np.asarray(forced, dtype=np.uint8)).cuda()))
     torch.cuda.synchronize()
     sb.sol_attn_bind_workspace(ws)

@@ -79,6 +79,20 @@ def _run_workload(name, n_extra=2, cross_check_density=None):
             out2, counts2, mask2, _ = hp.run_gpu(q, k, v, wl.block, beta, impl=sb.SOL_IMPL_MMA_SYNC, ws=ws)
             assert np.array_equal(mask2, mask) and torch.equal(counts2, counts)
             assert float((out2.float() - of).abs().max()) <= 2 * hp.MAX_ABS
+        # ---- the optional routing pre-pass in the same configuration: its decisions against the oracle on every
+        #      head, its outputs bit-identical to the in-kernel router's wherever the two routed alike
+        out_p, counts_p, mask_p, _ = hp.run_gpu(q, k, v, wl.block, beta, ws=ws, routing=sb.SOL_ROUTING_PREPASS)
+        counts_p = counts_p.cpu().numpy()
+        assert np.array_equal(counts_p, mask_p.sum(axis=-1))
+        pre_flips = 0
+        for h in range(H):
+            _, _, tau, ref_mask = routing[h].at(beta)
+            pre_flips += hp.check_mask(mask_p[0, h], counts_p[0, h], routing[h].s_hat, tau, ref_mask)["in_band_flips"]
+        same = ~(mask_p != mask).any(axis=-1)[0]                                   # [H, Nq]
+        rows_same = torch.from_numpy(np.repeat(same, wl.block, axis=1)[:, :N]).cuda()   # [H, N]
+        assert bool((out_p.view(torch.int16)[0] == out.view(torch.int16)[0])[rows_same].all())
+        pre_differ = int((~same).sum())
+        del out_p
         # ---- routing of every head against the oracle
         agg = {}
         flipped_heads = []
@@ -103,7 +117,8 @@ def _run_workload(name, n_extra=2, cross_check_density=None):
               f"{agg['blocks']}, flips {agg['in_band_flips']}; outputs on heads {heads} ({agg['tiles']} query blocks): "
               f"max-abs {agg['max_abs']:.2e}, over |ref|<2 {agg['max_abs_ref_lt_2']:.2e}, vs bf16-rounded oracle "
               f"{agg['max_abs_vs_bf16_oracle']:.2e}, elements over 1e-2: {agg['n_over_1e-2']}, rel-L2 {agg['rel_l2']:.2e}, "
-              f"max |ref| {agg['max_abs_out']:.2f}")
+              f"max |ref| {agg['max_abs_out']:.2f}; routing pre-pass: flips {pre_flips}, query blocks routed unlike the "
+              f"in-kernel router {pre_differ}, all others bit-identical")
     return wl, bits, (q, k, v), ws
 
 

@@ -45,12 +45,12 @@ def _small_problem(seed, B, H, N, d, structured=True):
 
 
 def _check_all_heads(bits, block, beta, impl, mode=None, mode_name="sol", scale=0.0, tiles=None,
-                     estimator="direct", forced=None):
+                     estimator="direct", forced=None, routing=0):
     qb, kb, vb = bits
     q, k, v = (hp.to_dev(x) for x in bits)
     mode = sb.SOL_MODE_SOL if mode is None else mode
     out, counts, mask, _ = hp.run_gpu(q, k, v, block, beta, mode=mode, impl=impl, scale=scale,
-                                      estimator=(1 if estimator == "diagonal" else 0), forced=forced)
+                                      estimator=(1 if estimator == "diagonal" else 0), forced=forced, routing=routing)
     B, H, N, d = q.shape
     out64 = hp.dev_to_f64(out)
     agg = {}
@@ -186,6 +186,69 @@ def test_tau_override_and_determinism(impl):
 
 
 # ----------------------------------------------------------------------------- host-side errors
+# ----------------------------------------------------------------------------- routing pre-pass
+@pytest.mark.parametrize("N,d,block", [(1000, 128, 128), (8329, 128, 128), (129, 128, 128), (1000, 64, 64),
+                                       (333, 128, 64), (2500, 64, 128)])
+def test_routing_prepass_matches_the_oracle(N, d, block):
+    """Eq. (4) evaluated by the pre-pass kernel: mask, counts and outputs against the oracle, like the in-kernel router."""
+    bits = _small_problem(N + d + 1, 2, 2, N, d)
+    agg = _check_all_heads(bits, block, 0.4, sb.SOL_IMPL_AUTO, routing=sb.SOL_ROUTING_PREPASS)
+    print("prepass", N, d, block, agg)
+
+
+def test_routing_prepass_agrees_with_the_fused_router():
+    """Same decisions as the in-kernel router outside the rounding band, hence the same outputs there; forced
+    blocks, the keep-or-drop mode and the degenerate thresholds go through the pre-pass too."""
+    wl = WORKLOADS["image"]
+    beta = load_betas()["image"][0.3]
+    bits = synth.generate(wl)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out_f, counts_f, mask_f, ws = hp.run_gpu(q, k, v, wl.block, beta)
+    out_p, counts_p, mask_p, _ = hp.run_gpu(q, k, v, wl.block, beta, ws=ws, routing=sb.SOL_ROUTING_PREPASS)
+    differ = mask_f != mask_p
+    print("prepass vs fused: differing decisions", int(differ.sum()), "of", mask_f.size)
+    assert differ.sum() <= 2                               # only pairs within rounding of the threshold
+    same_rows = ~differ.any(axis=-1)                       # [B, H, Nq]
+    of = out_f.view(torch.int16).cpu().numpy().reshape(wl.batch, wl.heads, -1, wl.block, wl.d)
+    op = out_p.view(torch.int16).cpu().numpy().reshape(wl.batch, wl.heads, -1, wl.block, wl.d)
+    assert np.array_equal(of[same_rows], op[same_rows])   # bit-identical where the routing is
+    assert np.array_equal(counts_p.cpu().numpy(), mask_p.sum(axis=-1))
+    agg = _check_all_heads(bits, wl.block, beta, sb.SOL_IMPL_AUTO, routing=sb.SOL_ROUTING_PREPASS)
+    print("prepass image", agg)
+    # forced blocks, keep-or-drop mode, select-all / select-none
+    small = _small_problem(23, 1, 2, 1500, 128)
+    forced = np.zeros(12, dtype=bool)
+    forced[[0, 5, 11]] = True
+    _check_all_heads(small, 128, 0.9, sb.SOL_IMPL_AUTO, forced=forced, routing=sb.SOL_ROUTING_PREPASS)
+    _check_all_heads(small, 128, 0.3, sb.SOL_IMPL_AUTO, mode=sb.SOL_MODE_EXACT_ONLY, mode_name="exact_only",
+                     routing=sb.SOL_ROUTING_PREPASS)
+    qs, ks, vs = (hp.to_dev(x) for x in small)
+    for beta_inf, want in ((-math.inf, 12), (math.inf, 0)):
+        _, counts, mask, _ = hp.run_gpu(qs, ks, vs, 128, beta_inf, routing=sb.SOL_ROUTING_PREPASS)
+        assert (counts.cpu().numpy() == want).all() and (mask.sum(axis=-1) == want).all()
+
+
+def test_routing_prepass_argument_rules():
+    bits = _small_problem(16, 1, 1, 256, 128)
+    q, k, v = (hp.to_dev(x) for x in bits)
+    out = torch.empty_like(q)
+    ws = sb.make_workspace(1, 1, 256, 128, 128, 128)
+    mask = torch.zeros(1, 1, 2, 1, dtype=torch.int32, device="cuda")
+    with pytest.raises(sb.SolAttnError) as e:              # the decisions need the caller's mask buffer
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.5, routing=sb.SOL_ROUTING_PREPASS)
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
+    with pytest.raises(sb.SolAttnError) as e:              # only the tcgen05 kernel reads them
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.5, routing=sb.SOL_ROUTING_PREPASS,
+                               mask_out=mask, impl=sb.SOL_IMPL_MMA_SYNC)
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, threshold=0.5, routing=7, mask_out=mask)
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
+    # dense mode has no routing: the option is ignored, no mask needed
+    sb.sol_attn_forward_ex(q, k, v, out, ws, 128, 128, mode=sb.SOL_MODE_DENSE, routing=sb.SOL_ROUTING_PREPASS)
+    torch.cuda.synchronize()
+
+
 def test_argument_validation():
     bits = _small_problem(15, 1, 1, 256, 128)
     q, k, v = (hp.to_dev(x) for x in bits)
