@@ -439,12 +439,15 @@ def main():
             qbar_c, kc_c = ws.qbar.contiguous(), ws.kc.contiguous()
             ms_thr_static = timed(lambda: sb.sol_attn_thresholds_static(qbar_c, kc_c, beta, mu_s, sg_s, tau_s),
                                   args.steps, 1)
-        routing = {"thresholds_ms": ms_thr, "thresholds_static_ms": ms_thr_static,
+        ms_mask = timed(lambda: sb.sol_attn_route_mask(B, H, N, d, wl.block, wl.block, mask_buf), args.steps, 1)
+        routing = {"thresholds_ms": ms_thr, "thresholds_static_ms": ms_thr_static, "mask_prepass_ms": ms_mask,
+                   "mask_prepass_bytes": int(mask_buf.numel() * 4),
                    "topk_ms": ms_topk, "topp_ms": ms_topp,
                    "topk_over_thresholds": ms_topk / ms_thr, "topp_over_thresholds": ms_topp / ms_thr,
                    "materialised_bytes": int(pmap.numel() * 4 + order.numel() * 4),
                    "note": "thresholds: mean, covariance and tau kernels on pooled data (nothing of size Nq x Nk "
-                           "exists); baselines: proxy map + routing indices in HBM, k = %d blocks, p = 0.9" % k_blocks}
+                           "exists); mask_prepass: the optional SOL_ROUTING_PREPASS kernel, one bit per block pair; baselines: "
+                           "proxy map + routing indices in HBM, k = %d blocks, p = 0.9" % k_blocks}
         check_status()
 
     # ---- accuracy ablation on the image workload (small): error against dense attention of the

@@ -150,6 +150,16 @@ sol_status_t sol_attn_forward(const void* q, const void* k, const void* v, void*
 sol_status_t sol_attn_dense(const void* q, const void* k, const void* v, void* out,
                             int B, int H, int N, int d, sol_stream_t stream);
 
+/* Routing decisions alone (the pre-pass of SOL_ROUTING_PREPASS): evaluates Eq. (4), s_ij > tau_i, for every
+ * (query block, key block) pair on the pooled tensors and thresholds a previous sol_attn_pool /
+ * sol_attn_thresholds / forward left in the bound workspace, and writes one bit per pair to `mask`
+ * (device, uint32 [B, H, Nq, ceil(Nk / 32)], bit j % 32 of word j / 32; caller-owned).  `tau_override`
+ * (device fp32 [B, H, Nq]) replaces the workspace's thresholds when not NULL; `forced_blocks` as in
+ * sol_attn_args.  `scale` <= 0 selects 1/sqrt(d).  One kernel on `stream`; does not synchronise. */
+sol_status_t sol_attn_route_mask(int B, int H, int N, int d, int block_q, int block_k, float scale,
+                                 const float* tau_override, const uint8_t* forced_blocks, uint32_t* mask,
+                                 sol_stream_t stream);
+
 /* Fully explicit variant: nothing is taken from the bound state. */
 typedef struct {
   const void* q; const void* k; const void* v;  /* device, bf16 [B,H,N,d]                       */

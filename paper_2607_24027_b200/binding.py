@@ -38,7 +38,7 @@ EXPORTS = [
     "sol_attn_bind_workspace", "sol_attn_pool", "sol_attn_forward", "sol_attn_dense",
     "sol_attn_forward_ex", "sol_attn_forward_host", "sol_attn_read_device_status",
     "sol_attn_launch_count", "sol_attn_thresholds_static", "sol_attn_thresholds_static_max_floats",
-    "sol_attn_route_materialized", "sol_attn_thresholds", "sol_attn_debug_set_wait",
+    "sol_attn_route_materialized", "sol_attn_thresholds", "sol_attn_debug_set_wait", "sol_attn_route_mask",
 ]
 
 
@@ -106,6 +106,8 @@ def lib() -> ctypes.CDLL:
     L.sol_attn_read_device_status.argtypes = [ctypes.c_void_p]
     L.sol_attn_launch_count.restype = ctypes.c_int64
     L.sol_attn_launch_count.argtypes = []
+    L.sol_attn_route_mask.restype = ctypes.c_int32
+    L.sol_attn_route_mask.argtypes = [ctypes.c_int] * 6 + [ctypes.c_float] + [ctypes.c_void_p] * 4
     L.sol_attn_thresholds_static.restype = ctypes.c_int32
     L.sol_attn_thresholds_static.argtypes = [ctypes.c_void_p] * 2 + [ctypes.c_int] * 5 + [ctypes.c_float] * 2 + \
                                             [ctypes.c_void_p] * 4
@@ -277,6 +279,13 @@ def sol_attn_thresholds(B, H, N, d, block_q, block_k, threshold, scale=0.0, esti
     """Recompute mu, sigma, tau in the bound workspace from the pooled tensors already there."""
     _check(lib().sol_attn_thresholds(B, H, N, d, block_q, block_k, float(threshold), float(scale), int(estimator),
                                      _stream(stream)), "sol_attn_thresholds")
+
+
+def sol_attn_route_mask(B, H, N, d, block_q, block_k, mask, scale=0.0, tau_override=None, forced_blocks=None, stream=None):
+    """Eq. (4) decisions of the bound workspace's pooled tensors and thresholds, one bit per block pair, into ``mask``
+    (int32 / uint32 [B, H, Nq, ceil(Nk / 32)])."""
+    _check(lib().sol_attn_route_mask(B, H, N, d, block_q, block_k, float(scale), _ptr(tau_override), _ptr(forced_blocks),
+                                     _ptr(mask), _stream(stream)), "sol_attn_route_mask")
 
 
 def sol_attn_route_materialized(qbar, kc, policy, param, proxy_map, tau, order=None, counts=None, scale=0.0,

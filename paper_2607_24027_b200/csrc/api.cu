@@ -192,6 +192,25 @@ sol_status_t sol_attn_thresholds(int B, int H, int N, int d, int block_q, int bl
   return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
 
+sol_status_t sol_attn_route_mask(int B, int H, int N, int d, int block_q, int block_k, float scale,
+                                 const float* tau_override, const uint8_t* forced_blocks, uint32_t* mask,
+                                 sol_stream_t stream) {
+  sol_status_t s = check_shape(B, H, N, d, block_q, block_k, false);
+  if (s != SOL_OK) return s;
+  if (!mask || std::isnan(scale) || std::isinf(scale)) return SOL_ERR_INVALID_ARG;
+  if (!g_bound.ws) return SOL_ERR_WORKSPACE;
+  if (g_bound.bytes < sol_attn_workspace_bytes(B, H, N, d, block_q, block_k)) return SOL_ERR_WORKSPACE;
+  if ((s = check_arch()) != SOL_OK) return s;
+  const sol::Problem p = make_problem(B, H, N, d, block_q, block_k, 0.f, scale, SOL_MODE_SOL, SOL_EST_MOMENTS,
+                                      forced_blocks);
+  const sol::WsPtrs ws = sol::make_ptrs(g_bound.ws, sol::make_layout(p.BH, p.Nq, p.Nk, p.d));
+  int n = 0;
+  const cudaError_t e = sol::launch_route_prepass(p, ws, tau_override ? tau_override : ws.tau, mask,
+                                                  static_cast<cudaStream_t>(stream), &n);
+  g_launches += n;
+  return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+}
+
 // keep_status: a later piece of one logical call must not wipe the device status of an earlier one
 static sol_status_t forward_impl(const sol_attn_args* a, bool keep_status) {
   if (!a) return SOL_ERR_INVALID_ARG;

@@ -215,6 +215,17 @@ def test_routing_prepass_agrees_with_the_fused_router():
     assert np.array_equal(counts_p.cpu().numpy(), mask_p.sum(axis=-1))
     agg = _check_all_heads(bits, wl.block, beta, sb.SOL_IMPL_AUTO, routing=sb.SOL_ROUTING_PREPASS)
     print("prepass image", agg)
+    # the pre-pass as an entry point of its own (bound workspace) writes the same bits
+    sb.sol_attn_bind_workspace(ws)
+    alone = torch.zeros(wl.batch, wl.heads, wl.n_blocks, sb.mask_words(wl.n_blocks), dtype=torch.int32, device="cuda")
+    launches = sb.sol_attn_launch_count()
+    sb.sol_attn_route_mask(wl.batch, wl.heads, wl.seq_len, wl.d, wl.block, wl.block, alone)
+    torch.cuda.synchronize()
+    assert sb.sol_attn_launch_count() == launches + 1
+    assert np.array_equal(hp.unpack_mask(alone, wl.n_blocks), mask_p)
+    with pytest.raises(sb.SolAttnError) as e:
+        sb.sol_attn_route_mask(wl.batch, wl.heads, wl.seq_len, wl.d, wl.block, wl.block, None)
+    assert e.value.status == sb.SOL_ERR_INVALID_ARG
     # forced blocks, keep-or-drop mode, select-all / select-none
     small = _small_problem(23, 1, 2, 1500, 128)
     forced = np.zeros(12, dtype=bool)
