@@ -2,7 +2,7 @@
 """Benchmark of the Sol-Attn fused forward path on synthetic video-DiT-shaped inputs.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload video720] [--density 0.15] [--no-sweep]
+                    [--workload video720] [--density 0.15] [--no-sweep] [--routing fused|prepass]
 
 One "step" is one pass of the whole hot path (pooling pre-pass, thresholds, fused kernel) over
 one batch (B=1, H=40, N=75600, d=128, block 128 for the default workload).  Prints ONE JSON line.
@@ -15,7 +15,8 @@ one batch (B=1, H=40, N=75600, d=128, block 128 for the default workload).  Prin
 * roofline: the fused kernel alone (``skip_pool``), computed FLOPs (exact pairs actually routed +
   the approximate outer loop) per launch / CUDA-event time, against the measured bf16 peak.
 * cpu_baseline: the CPU oracle timed on a bounded sample of the same workload.
-* sweep: every density of the workload's threshold sweep plus the dense-mode run.
+* sweep: every density of the workload's threshold sweep plus the dense-mode run; every routed point also with the
+  optional routing pre-pass (``routing_prepass``).  ``--routing prepass`` takes the headline numbers that way too.
 
 Under torchrun ONE call is sharded by heads: rank r generates and processes only its own contiguous
 range of the workload's heads (heads are independent; there is no collective on the data path), timing
@@ -247,6 +248,8 @@ def main():
     ap.add_argument("--workload", default="video720", choices=list(WORKLOADS))
     ap.add_argument("--density", type=float, default=0.15)
     ap.add_argument("--kernel", default="auto", choices=["auto", "tcgen05", "mma_sync"])
+    ap.add_argument("--routing", default="fused", choices=["fused", "prepass"],
+                    help="where Eq. (4) is decided for the headline numbers: inside the fused kernel (the paper's structure, default) or by the optional pre-pass kernel")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--heads", type=int, default=0, help="override the head count (profiling small cases)")
@@ -332,9 +335,13 @@ def main():
             raise SystemExit(f"device status {sb.status_string(st)}")
 
     def full_step(b=beta):
+        if args.routing == "prepass":
+            return prepass_step(b)
         sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl)
 
     def kernel_only(b=beta):
+        if args.routing == "prepass":
+            return prepass_step(b, True)
         sb.sol_attn_forward_ex(q, k, v, out, ws, wl.block, wl.block, threshold=b, impl=impl, skip_pool=True)
 
     mask_buf = torch.zeros(B, H, wl.n_blocks, sb.mask_words(wl.n_blocks), dtype=torch.int32, device="cuda")
@@ -481,7 +488,7 @@ def main():
         "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"{wl.name} density {args.density}", "B": B, "H": H, "N": N, "d": d,
-                   "block": wl.block, "beta": beta, "achieved_density": density, "kernel": args.kernel,
+                   "block": wl.block, "beta": beta, "achieved_density": density, "kernel": args.kernel, "routing": args.routing,
                    "l2": "inputs (3 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
                    "parallelism": ("single GPU" if world == 1 else "replicas (no collective)" if args.replicas else
                                    f"one call sharded by heads: {H} of {wl.batch * wl.heads} heads on this rank, "
